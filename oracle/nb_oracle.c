@@ -1,0 +1,68 @@
+/*
+ * CPU oracle for the dense linear layers (forward and backward) of the GPT-2
+ * 124M training step. TEST INFRASTRUCTURE ONLY: plain, slow, and independent of
+ * the CUDA library. Only the tests, the smoke check and the benchmark's CPU
+ * baseline may load it.
+ *
+ * Two instances of the same source: suffix _f32 computes and accumulates in
+ * float (the arithmetic the training step's precision statement names), suffix
+ * _f64 in double (used to bound the float instance's own rounding and as the
+ * parity reference). See nb_oracle_impl.inc for the definitions followed.
+ *
+ * Every exported function is pinned by tests that do not use this file:
+ * library GELU/SiLU, library autograd, integer-exact products, finite
+ * differences and adjoint identities.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define NBO_ACT_NONE 0
+#define NBO_ACT_GELU 1
+#define NBO_ACT_SWIGLU 2
+
+#define REAL float
+#define SUFFIX _f32
+#define TANH tanhf
+#define EXP expf
+#include "nb_oracle_impl.inc"
+#undef REAL
+#undef SUFFIX
+#undef TANH
+#undef EXP
+
+#define REAL double
+#define SUFFIX _f64
+#define TANH tanh
+#define EXP exp
+#include "nb_oracle_impl.inc"
+#undef REAL
+#undef SUFFIX
+#undef TANH
+#undef EXP
+
+/* Column sum used by the stand-alone dbias reduction: dbias[o] (+)= sum_m dout[m,o]. */
+int nbo_reduce_dbias_f64(double *dbias, const float *dout, int64_t BT, int64_t OC, int accumulate)
+{
+    if (!dbias || !dout || BT < 0 || OC < 0) return -1;
+    for (int64_t o = 0; o < OC; ++o) {
+        double s = 0.0;
+        for (int64_t m = 0; m < BT; ++m) s += (double)dout[m * OC + o];
+        if (accumulate)
+            dbias[o] += s;
+        else
+            dbias[o] = s;
+    }
+    return 0;
+}
+
+int nbo_num_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,179 @@
+/*
+ * nb_linear: dense bf16 linear layers, forward and backward, for NVIDIA B200 (sm_100a).
+ *
+ * The calls below are the part of a GPT-2 124M training step that takes most of its
+ * time: the QKV, attention-output, MLP fc (+GELU), MLP projection and tied lm_head
+ * products, forward and backward (paper: Results/Speed, the stage table: "GEMMs
+ * (projections and head)"; layer shapes in Method/Model and Figure 1). The library
+ * follows the paper's description of a C ABI that bindings in any language compose
+ * from, with return codes that tell a malformed request from a failed execution
+ * (paper: The stack under test).
+ *
+ * Conventions for every call
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned,
+ *    row-major and dense. The library never frees or keeps caller memory.
+ *  - Activations, weights, biases and activation gradients are bf16. Weight and bias
+ *    gradients are fp32 (paper: Method/Optimisation and precision). Products are
+ *    accumulated in fp32 on the tensor cores; each bf16 result is rounded once,
+ *    round-to-nearest-even.
+ *  - Shapes: inp [BT, C], weight [OC, C], bias [OC], out / dout [BT, OC]
+ *    ([BT, OC/2] for SwiGLU), pre_act [BT, OC], dinp [BT, C], dweight [OC, C],
+ *    dbias [OC]. C and OC must be multiples of 8 (OC/2 a multiple of 8 for SwiGLU);
+ *    BT is arbitrary. Dimensions must be below 2^31 and BT*OC, BT*C below 2^40.
+ *  - Calls are asynchronous on a CUDA stream: the `_ex` forms take it as an argument
+ *    (a cudaStream_t passed as void*), the short forms use the stream last given to
+ *    nb_set_stream on the calling thread (default: the legacy default stream).
+ *  - Return value: NB_OK or an NB_ERR_* code; nb_last_error() gives the text for the
+ *    calling thread. NB_ERR_INVALID_ARG and NB_ERR_UNSUPPORTED are malformed requests
+ *    and launch nothing. NB_ERR_CUDA is a driver / launch failure. NB_ERR_TIMEOUT is
+ *    reported by nb_check_status when a kernel gave up on a bounded wait.
+ *  - The library keeps a grow-only device workspace (only for backward calls that
+ *    apply this layer's own activation derivative, see below), a 64-byte device status
+ *    word per device and a host-side cache of TMA descriptors.
+ */
+#ifndef NB_LINEAR_H
+#define NB_LINEAR_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NB_OK 0
+#define NB_ERR_INVALID_ARG 1 /* null / misaligned pointer, negative size, bad enum */
+#define NB_ERR_UNSUPPORTED 2 /* shape outside the constraints above */
+#define NB_ERR_CUDA 3        /* CUDA driver or launch failure */
+#define NB_ERR_TIMEOUT 4     /* a device-side bounded wait expired */
+
+#define NB_ACT_NONE 0
+#define NB_ACT_GELU 1   /* tanh form: 0.5 z (1 + tanh(sqrt(2/pi)(z + 0.044715 z^3))) */
+#define NB_ACT_SWIGLU 2 /* weight rows [0,H) gate, [H,2H) up; out = silu(gate) * up */
+
+#define NB_DTYPE_F32 0
+#define NB_DTYPE_BF16 1
+
+/* Library version as major*10000 + minor*100 + patch. */
+int nb_version(void);
+
+/* Text of the last error on the calling thread ("" if none). Never NULL. */
+const char *nb_last_error(void);
+
+/* Stream used by the short-form calls on this thread (a cudaStream_t; NULL = default). */
+int nb_set_stream(void *stream);
+void *nb_get_stream(void);
+
+/*
+ * Number of bf16 elements the `out` argument of nb_linear_forward must hold:
+ * BT*OC for NB_ACT_NONE; BT*OC (activated plane) + BT*OC (pre-activation plane) for
+ * NB_ACT_GELU; BT*OC/2 + BT*OC for NB_ACT_SWIGLU. Returns -1 on a bad argument.
+ */
+int64_t nb_linear_out_elems(int64_t BT, int64_t OC, int act);
+
+/*
+ * Forward: z = inp . weight^T (+ bias); out = act(z).
+ * (paper: Figure 1, "768 -> 3072, GELU, 3072 -> 768"; head tied and bias-free)
+ *
+ *   out     [out] act == NONE : [BT, OC] bf16.
+ *                 act != NONE : two planes back to back, the activated result first
+ *                 ([BT, OC], or [BT, OC/2] for SwiGLU) and then the pre-activation z
+ *                 [BT, OC], which backward needs. Size: nb_linear_out_elems().
+ *   inp     [in]  [BT, C] bf16
+ *   weight  [in]  [OC, C] bf16
+ *   bias    [in]  [OC] bf16 or NULL
+ *   act           NB_ACT_*
+ * BT == 0 is accepted and does nothing.
+ */
+int nb_linear_forward(void *out, const void *inp, const void *weight, const void *bias,
+                      int64_t BT, int64_t C, int64_t OC, int act);
+
+/*
+ * Forward with the pre-activation plane and the stream given explicitly.
+ * pre_act: [BT, OC] bf16, written when act != NONE (may be NULL to skip storing it;
+ * must be NULL or ignored for act == NONE). nb_linear_forward wraps this call.
+ */
+int nb_linear_forward_ex(void *out, void *pre_act, const void *inp, const void *weight,
+                         const void *bias, int64_t BT, int64_t C, int64_t OC, int act,
+                         void *stream);
+
+/*
+ * Backward of one layer (paper: Method/Optimisation and precision for the fp32
+ * gradients; Method/Batch geometry for accumulation over micro-steps).
+ *
+ *   dz      = dout                      when pre_act == NULL
+ *           = dout * gelu'(pre_act)     when pre_act != NULL (this layer's own
+ *                                       pre-activation [BT, OC]; tanh-GELU)
+ *   dinp    [out] [BT, C] bf16  = dz . weight              always overwritten
+ *   dweight [i/o] [OC, C] fp32 (+)= dz^T . inp
+ *   dbias   [i/o] [OC]    fp32 (+)= column sums of dz
+ *   accumulate    0: dweight and dbias are overwritten (they need not be zeroed);
+ *                 non-zero: the new gradient is added to what they hold.
+ * Any of dinp, dweight, dbias may be NULL; that product is skipped (frozen weights).
+ * inp may be NULL when dweight is NULL; weight may be NULL when dinp is NULL.
+ * BT == 0: dinp untouched, dweight/dbias zeroed when accumulate == 0.
+ *
+ * When pre_act != NULL, dz is first written to the library's device workspace
+ * (BT*OC bf16, allocated on first need with cudaMalloc and kept). Summation order of
+ * dweight/dbias across row blocks is not fixed, so results may differ in the last
+ * bits between runs.
+ */
+int nb_linear_backward(void *dinp, void *dweight, void *dbias, const void *dout,
+                       const void *inp, const void *weight, const void *pre_act, int64_t BT,
+                       int64_t C, int64_t OC, int accumulate);
+
+/*
+ * Backward, general form.
+ *   act           activation of THIS layer, applied through pre_act (required when
+ *                 act != NONE): GELU as above; SWIGLU with dout [BT, OC/2] and
+ *                 pre_act [BT, OC] = [gate | up]:
+ *                   dz[:, j]     = dout[:, j] * up_j * silu'(gate_j)
+ *                   dz[:, H + j] = dout[:, j] * silu(gate_j)
+ *   inp_pre_act   NULL, or [BT, C] bf16: the pre-activation of the GELU layer that
+ *                 produced `inp`. Then dinp = (dz . weight) * gelu'(inp_pre_act), i.e.
+ *                 the dz of that producer, applied in the dgrad epilogue in fp32
+ *                 before the single rounding to bf16 (the activation backward the
+ *                 paper's stack launches as a separate kernel, fused here).
+ *   dweight_dtype NB_DTYPE_F32 (the paper's arrangement). NB_DTYPE_BF16 is accepted
+ *                 only with accumulate == 0.
+ *   stream        cudaStream_t as void*.
+ */
+int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *dout,
+                          const void *inp, const void *weight, const void *pre_act,
+                          const void *inp_pre_act, int64_t BT, int64_t C, int64_t OC, int act,
+                          int accumulate, int dweight_dtype, void *stream);
+
+/*
+ * Stand-alone column reduction: dbias[o] (+)= sum over rows of dout[m, o].
+ * dout [BT, OC] bf16, dbias [OC] fp32, OC a multiple of 8. Uses the stream of
+ * nb_set_stream. (The bias gradient of every biased layer; paper: Method/Model lists
+ * the biased linears through the parameter count.)
+ */
+int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int accumulate);
+
+/*
+ * Make sure the workspace holds at least `bytes` (so later calls do not allocate), or
+ * release everything the library holds on the current device (workspace, status word,
+ * descriptor cache) with nb_release.
+ */
+int nb_workspace_reserve(int64_t bytes);
+int nb_release(void);
+
+/*
+ * Synchronise the current device and report whether any kernel since the last check
+ * gave up on a bounded wait (NB_ERR_TIMEOUT, detail in nb_last_error) or a CUDA error is
+ * pending (NB_ERR_CUDA). Clears the device status word.
+ */
+int nb_check_status(void);
+
+/*
+ * Self-test of the bounded-wait mechanism: launches a one-block kernel that waits, for
+ * at most `limit_us` microseconds, on a barrier nothing ever signals, then returns
+ * normally after recording the expiry. nb_check_status() afterwards reports
+ * NB_ERR_TIMEOUT; the context stays usable.
+ */
+int nb_debug_wait_timeout(int64_t limit_us);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NB_LINEAR_H */

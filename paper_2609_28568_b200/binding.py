@@ -1,0 +1,173 @@
+"""ctypes binding of the nb_linear C ABI: argument marshalling only.
+
+Functions named like the C entry points take torch CUDA tensors (or raw device
+pointers as ints) and pass pointers and sizes straight through; every step of
+the computation runs in the CUDA library. There is no CPU path: if the library
+has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+NB_OK, NB_ERR_INVALID_ARG, NB_ERR_UNSUPPORTED, NB_ERR_CUDA, NB_ERR_TIMEOUT = 0, 1, 2, 3, 4
+ACT_NONE, ACT_GELU, ACT_SWIGLU = 0, 1, 2
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+EXPORTS = (
+    "nb_version", "nb_last_error", "nb_set_stream", "nb_get_stream", "nb_linear_out_elems",
+    "nb_linear_forward", "nb_linear_forward_ex", "nb_linear_backward", "nb_linear_backward_ex",
+    "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
+    "nb_debug_wait_timeout",
+)
+
+_lib = None
+_vp, _i64, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+
+
+class NbError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"nb_linear error {code}: {msg}")
+        self.code = code
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library. Raises if it was never built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2609_28568_b200.build` "
+                "(the CUDA library is the only implementation)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.nb_version.restype = _int
+        L.nb_last_error.restype = ctypes.c_char_p
+        L.nb_set_stream.argtypes = [_vp]
+        L.nb_get_stream.restype = _vp
+        L.nb_linear_out_elems.argtypes = [_i64, _i64, _int]
+        L.nb_linear_out_elems.restype = _i64
+        L.nb_linear_forward.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _int]
+        L.nb_linear_forward_ex.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _int, _vp]
+        L.nb_linear_backward.argtypes = [_vp] * 7 + [_i64, _i64, _i64, _int]
+        L.nb_linear_backward_ex.argtypes = [_vp] * 8 + [_i64, _i64, _i64, _int, _int, _int, _vp]
+        L.nb_reduce_dbias.argtypes = [_vp, _vp, _i64, _i64, _int]
+        L.nb_workspace_reserve.argtypes = [_i64]
+        L.nb_debug_wait_timeout.argtypes = [_i64]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _check(rc: int) -> None:
+    if rc != NB_OK:
+        raise NbError(rc, lib().nb_last_error().decode())
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def nb_version() -> int:
+    return lib().nb_version()
+
+
+def nb_last_error() -> str:
+    return lib().nb_last_error().decode()
+
+
+def nb_linear_out_elems(BT: int, OC: int, act: int) -> int:
+    return lib().nb_linear_out_elems(BT, OC, act)
+
+
+def nb_set_stream(stream) -> None:
+    _check(lib().nb_set_stream(stream))
+
+
+def nb_linear_forward(out, inp, weight, bias, BT, C, OC, act) -> None:
+    """Short form: `out` holds the activated plane followed by the pre-activation plane."""
+    lib().nb_set_stream(_stream())
+    _check(lib().nb_linear_forward(_ptr(out), _ptr(inp), _ptr(weight), _ptr(bias), BT, C, OC, act))
+
+
+def nb_linear_forward_ex(out, pre_act, inp, weight, bias, BT, C, OC, act, stream=None) -> None:
+    _check(lib().nb_linear_forward_ex(_ptr(out), _ptr(pre_act), _ptr(inp), _ptr(weight), _ptr(bias),
+                                      BT, C, OC, act, _stream() if stream is None else stream))
+
+
+def nb_linear_backward(dinp, dweight, dbias, dout, inp, weight, pre_act, BT, C, OC, accumulate) -> None:
+    lib().nb_set_stream(_stream())
+    _check(lib().nb_linear_backward(_ptr(dinp), _ptr(dweight), _ptr(dbias), _ptr(dout), _ptr(inp),
+                                    _ptr(weight), _ptr(pre_act), BT, C, OC, int(accumulate)))
+
+
+def nb_linear_backward_ex(dinp, dweight, dbias, dout, inp, weight, pre_act, inp_pre_act, BT, C, OC,
+                          act, accumulate, dweight_dtype=DTYPE_F32, stream=None) -> None:
+    _check(lib().nb_linear_backward_ex(_ptr(dinp), _ptr(dweight), _ptr(dbias), _ptr(dout), _ptr(inp),
+                                       _ptr(weight), _ptr(pre_act), _ptr(inp_pre_act), BT, C, OC, act,
+                                       int(accumulate), dweight_dtype,
+                                       _stream() if stream is None else stream))
+
+
+def nb_reduce_dbias(dbias, dout, BT, OC, accumulate) -> None:
+    lib().nb_set_stream(_stream())
+    _check(lib().nb_reduce_dbias(_ptr(dbias), _ptr(dout), BT, OC, int(accumulate)))
+
+
+def nb_workspace_reserve(nbytes: int) -> None:
+    _check(lib().nb_workspace_reserve(nbytes))
+
+
+def nb_release() -> None:
+    _check(lib().nb_release())
+
+
+def nb_check_status() -> None:
+    """Synchronise and raise NbError(NB_ERR_TIMEOUT / NB_ERR_CUDA) if a kernel reported a failure."""
+    _check(lib().nb_check_status())
+
+
+def nb_debug_wait_timeout(limit_us: int) -> None:
+    lib().nb_set_stream(_stream())
+    _check(lib().nb_debug_wait_timeout(limit_us))
+
+
+# ------------------------------------------------------------------ conveniences (allocation only)
+
+def linear_forward(inp, weight, bias=None, act=ACT_NONE):
+    """Allocate the outputs and call nb_linear_forward_ex. Returns (out, pre_act or None)."""
+    BT, C = inp.shape
+    OC = weight.shape[0]
+    ocols = OC // 2 if act == ACT_SWIGLU else OC
+    out = torch.empty((BT, ocols), dtype=torch.bfloat16, device=inp.device)
+    pre = torch.empty((BT, OC), dtype=torch.bfloat16, device=inp.device) if act != ACT_NONE else None
+    nb_linear_forward_ex(out, pre, inp, weight, bias, BT, C, OC, act)
+    return out, pre
+
+
+def linear_backward(dout, inp, weight, pre_act=None, inp_pre_act=None, act=ACT_NONE, dweight=None,
+                    dbias=None, accumulate=False, need_dinp=True, need_dweight=True,
+                    need_dbias=True):
+    """Allocate missing outputs and call nb_linear_backward_ex. Returns (dinp, dweight, dbias)."""
+    BT = dout.shape[0]
+    OC, C = weight.shape
+    dev = dout.device
+    dinp = torch.empty((BT, C), dtype=torch.bfloat16, device=dev) if need_dinp else None
+    if need_dweight and dweight is None:
+        dweight = torch.empty((OC, C), dtype=torch.float32, device=dev)
+    if need_dbias and dbias is None:
+        dbias = torch.empty((OC,), dtype=torch.float32, device=dev)
+    nb_linear_backward_ex(dinp, dweight if need_dweight else None, dbias if need_dbias else None,
+                          dout, inp, weight, pre_act, inp_pre_act, BT, C, OC, act, accumulate)
+    return dinp, dweight, dbias

@@ -1,0 +1,143 @@
+// HBM-bound helper kernels around the GEMMs: activation backward (dz), the stand-alone dbias
+// column reduction, and the bounded-wait self-test.
+#pragma once
+#include "gemm_sm100.cuh"
+
+namespace nb {
+
+__device__ __forceinline__ float silu_bwd(float g)
+{
+    const float s = __fdividef(1.0f, 1.0f + __expf(-g));
+    return s * (1.0f + g * (1.0f - s));
+}
+
+// dz = dout * gelu'(pre), 8 bf16 per thread per iteration (128-bit loads and stores).
+__global__ void __launch_bounds__(256)
+gelu_backward_kernel(uint4 *__restrict__ dz, const uint4 *__restrict__ dout,
+                     const uint4 *__restrict__ pre, long long nvec)
+{
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < nvec;
+         i += stride) {
+        const uint4 d = __ldg(dout + i);
+        const uint4 x = __ldg(pre + i);
+        const uint32_t dv[4] = {d.x, d.y, d.z, d.w};
+        const uint32_t xv[4] = {x.x, x.y, x.z, x.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float lo = ptx::bf16_lo(dv[k]) * gelu_bwd(ptx::bf16_lo(xv[k]));
+            const float hi = ptx::bf16_hi(dv[k]) * gelu_bwd(ptx::bf16_hi(xv[k]));
+            o[k] = ptx::pack_bf16x2(lo, hi);
+        }
+        dz[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// SwiGLU backward: dout [BT, H], pre [BT, 2H] = [gate | up]  ->  dz [BT, 2H].
+//   dz[:, j] = dout * up * silu'(gate) ; dz[:, H + j] = dout * silu(gate)
+__global__ void __launch_bounds__(256)
+swiglu_backward_kernel(uint4 *__restrict__ dz, const uint4 *__restrict__ dout,
+                       const uint4 *__restrict__ pre, long long BT, int hvec /* H / 8 */)
+{
+    const long long total = BT * hvec;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += stride) {
+        const long long m = i / hvec;
+        const int j = static_cast<int>(i - m * hvec);
+        const uint4 d = __ldg(dout + i);
+        const uint4 g = __ldg(pre + m * 2 * hvec + j);
+        const uint4 u = __ldg(pre + m * 2 * hvec + hvec + j);
+        const uint32_t dv[4] = {d.x, d.y, d.z, d.w};
+        const uint32_t gv[4] = {g.x, g.y, g.z, g.w};
+        const uint32_t uv[4] = {u.x, u.y, u.z, u.w};
+        uint32_t og[4], ou[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float d0 = ptx::bf16_lo(dv[k]), d1 = ptx::bf16_hi(dv[k]);
+            const float g0 = ptx::bf16_lo(gv[k]), g1 = ptx::bf16_hi(gv[k]);
+            const float u0 = ptx::bf16_lo(uv[k]), u1 = ptx::bf16_hi(uv[k]);
+            og[k] = ptx::pack_bf16x2(d0 * u0 * silu_bwd(g0), d1 * u1 * silu_bwd(g1));
+            ou[k] = ptx::pack_bf16x2(d0 * silu_fwd(g0), d1 * silu_fwd(g1));
+        }
+        dz[m * 2 * hvec + j] = make_uint4(og[0], og[1], og[2], og[3]);
+        dz[m * 2 * hvec + hvec + j] = make_uint4(ou[0], ou[1], ou[2], ou[3]);
+    }
+}
+
+// dbias[o] += sum over a block of rows of dz[m, o].
+// A block owns 128 columns and `rows_per_block` rows. Inside a warp, lanes 0..7 hold eight
+// 128-bit column vectors (64 columns) and the lane's upper bits select one of four rows, for two
+// 64-column halves; rows are summed in registers, then across the four row lanes by shuffles,
+// across the eight warps through shared memory, and across blocks by atomic adds.
+constexpr int kDbiasCols = 128;
+constexpr int kDbiasThreads = 256;
+
+__global__ void __launch_bounds__(kDbiasThreads)
+dbias_kernel(float *__restrict__ dbias, const __nv_bfloat16 *__restrict__ dz, long long BT, int OC,
+             int rows_per_block)
+{
+    __shared__ float part[8][kDbiasCols];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cv = lane & 7;   // column vector inside a 64-column half
+    const int rs = lane >> 3;  // row inside a group of four
+    const int col0 = blockIdx.x * kDbiasCols;
+    const long long r_begin = static_cast<long long>(blockIdx.y) * rows_per_block;
+    const long long r_end = min(r_begin + rows_per_block, BT);
+    float acc[2][8];
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[h][k] = 0.0f;
+    const bool in0 = col0 + cv * 8 < OC;
+    const bool in1 = col0 + 64 + cv * 8 < OC;
+    for (long long r = r_begin + warp * 4 + rs; r < r_end; r += 32) {
+        const __nv_bfloat16 *rowp = dz + r * OC + col0 + cv * 8;
+        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = make_uint4(0, 0, 0, 0);
+        if (in0) v0 = __ldg(reinterpret_cast<const uint4 *>(rowp));
+        if (in1) v1 = __ldg(reinterpret_cast<const uint4 *>(rowp + 64));
+        const uint32_t a[4] = {v0.x, v0.y, v0.z, v0.w};
+        const uint32_t b[4] = {v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc[0][2 * k] += ptx::bf16_lo(a[k]);
+            acc[0][2 * k + 1] += ptx::bf16_hi(a[k]);
+            acc[1][2 * k] += ptx::bf16_lo(b[k]);
+            acc[1][2 * k + 1] += ptx::bf16_hi(b[k]);
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            float v = acc[h][k];
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            if (rs == 0) part[warp][h * 64 + cv * 8 + k] = v;
+        }
+    __syncthreads();
+    if (threadIdx.x < kDbiasCols) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
+        const int col = col0 + threadIdx.x;
+        if (col < OC) atomicAdd(dbias + col, s);
+    }
+}
+
+// Waits on a barrier that nothing signals, for at most limit_ns, then leaves normally.
+__global__ void wait_timeout_kernel(int *status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+        const WaitCtx w{ptx::smem_u32(&abort_flag), status, limit_ns};
+        (void)wait_barrier(w, ptx::smem_u32(&bar), 0, 900);
+    }
+}
+
+}  // namespace nb

@@ -1,0 +1,598 @@
+// Persistent, warp-specialised bf16 GEMM for sm_100a:  D[M,N] = sum_k A[m,k] * B[n,k]
+//
+//   warp 0      TMA producer: fills a ring of shared-memory stages (A tile 128x64, B tile Nx64)
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (128 x BLOCK_N x 16) into TMEM;
+//               two accumulators so the next tile's main loop overlaps this tile's epilogue
+//   warps 2..5  epilogue: tcgen05.ld -> fp32 registers -> bias / activation -> swizzled
+//               shared staging -> TMA store (or TMA reduce-add for split-K fp32 results)
+//
+// Operand layouts. "K-major" means the reduction index is contiguous in global memory (forward:
+// both operands). "MN-major" means the output index is contiguous (dgrad reads the weight as
+// B[n=c, k=o] from W[o, c]; wgrad reads dz and inp as A[m=o, k=row], B[n=c, k=row]); those tiles
+// are fetched as 64(k) x 64(mn) boxes and described to the tensor core as MN-major, so no
+// transpose is ever materialised.
+//
+// Every wait on an mbarrier is bounded in time; on expiry the kernel records the event in the
+// status word, stops issuing work, and all threads leave through the common exit.
+#pragma once
+#include "ptx.cuh"
+
+namespace nb {
+
+constexpr int kBlockM = 128;
+constexpr int kBlockK = 64;   // bf16 elements per stage along K = one 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kNumThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr uint32_t kStgBytes = 16384;  // one staging buffer: 128 rows x 128 bytes
+constexpr int kStatusTimeout = 4;      // == NB_ERR_TIMEOUT
+constexpr int kStatusBadSmem = 5;
+
+enum EpiMode : int {
+    kEpiStore = 0,        // D(bf16) = acc (+ bias)
+    kEpiGelu = 1,         // E(bf16) = z = acc + bias ; D(bf16) = gelu(z)
+    kEpiSwiglu = 2,       // E = z (gate | up planes) ; D[:, j] = silu(gate_j) * up_j
+    kEpiMulGeluGrad = 3,  // D(bf16) = acc * gelu'(E)    (E is read)
+    kEpiF32 = 4           // D(fp32) = acc, stored or reduce-added
+};
+
+struct GemmParams {
+    int M, N, K;
+    int tiles_m, tiles_n;
+    int splits;             // split-K factor (kEpiF32), else 1
+    int kblocks_per_split;  // 64-wide k blocks handled by one unit
+    int kblocks;            // ceil(K / 64)
+    int group_m;            // rasterisation: m-tiles per group
+    int swiglu_h;           // kEpiSwiglu: H (gate rows [0,H), up rows [H,2H) of B)
+    int reduce;             // kEpiF32: 1 reduce-add into D, 0 overwrite
+    const __nv_bfloat16 *bias;  // [N] or nullptr
+    int *status;
+    unsigned long long timeout_ns;
+};
+
+template <int BLOCK_N_, int STAGES_, int NSTG_, bool A_MN_, bool B_MN_, int EPI_>
+struct GemmCfg {
+    static constexpr int BLOCK_N = BLOCK_N_;
+    static constexpr int STAGES = STAGES_;
+    static constexpr int NSTG = NSTG_;
+    static constexpr bool A_MN = A_MN_;
+    static constexpr bool B_MN = B_MN_;
+    static constexpr int EPI = EPI_;
+    static constexpr uint32_t A_BYTES = kBlockM * kBlockK * 2;
+    static constexpr uint32_t B_BYTES = BLOCK_N * kBlockK * 2;
+    static constexpr uint32_t OFF_A = 0;
+    static constexpr uint32_t OFF_B = STAGES * A_BYTES;
+    static constexpr uint32_t OFF_STG = STAGES * (A_BYTES + B_BYTES);
+    static constexpr uint32_t OFF_BIAS = OFF_STG + NSTG * kStgBytes;
+    static constexpr uint32_t OFF_BAR = OFF_BIAS + BLOCK_N * 4;
+    static constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+    static constexpr uint32_t TMEM_COLS = (2 * BLOCK_N <= 32) ? 32
+                                          : (2 * BLOCK_N <= 64) ? 64
+                                          : (2 * BLOCK_N <= 128) ? 128
+                                          : (2 * BLOCK_N <= 256) ? 256 : 512;
+    // staging buffers used by one epilogue step, and steps per tile
+    static constexpr int BUFS_PER_STEP = (EPI == kEpiGelu) ? 2 : (EPI == kEpiSwiglu) ? 3 : 1;
+    static constexpr int SLOTS = NSTG / BUFS_PER_STEP;
+    static constexpr int STEPS = (EPI == kEpiF32) ? BLOCK_N / 32
+                                 : (EPI == kEpiSwiglu) ? BLOCK_N / 128 : BLOCK_N / 64;
+    static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
+    static_assert(2 * BLOCK_N <= 512, "two accumulators must fit in TMEM");
+    static_assert(NSTG % BUFS_PER_STEP == 0 && SLOTS >= 1, "staging ring");
+    static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 3, "aux prefetch needs a ring of >= 3");
+    static_assert(EPI != kEpiSwiglu || BLOCK_N == 256, "SwiGLU tiles pair 128 gate + 128 up cols");
+    static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+};
+
+// barrier slots inside the 256-byte barrier region (8 bytes each)
+//   [0, S)      full[s]     TMA -> MMA
+//   [S, 2S)     empty[s]    MMA -> TMA
+//   2S, 2S+1    tmem_full   MMA -> epilogue
+//   2S+2, 2S+3  tmem_empty  epilogue -> MMA
+//   2S+4 .. +7  aux_full    TMA -> epilogue (kEpiMulGeluGrad)
+//   byte 240: TMEM base address, 244: abort flag (any role), 248: epilogue abort flag
+
+struct WaitCtx {
+    uint32_t abort_addr;
+    int *status;
+    unsigned long long timeout_ns;
+};
+
+__device__ __forceinline__ bool wait_barrier(const WaitCtx &w, uint32_t bar, uint32_t parity,
+                                             int where)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = ptx::globaltimer_ns();
+    uint32_t it = 0;
+    while (true) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((++it & 15u) == 0) {
+            if (ptx::ld_shared_u32_volatile(w.abort_addr) != 0) return false;
+            if (ptx::globaltimer_ns() - t0 > w.timeout_ns) {
+                ptx::st_shared_u32_volatile(w.abort_addr, 1);
+                if (atomicCAS(w.status, 0, kStatusTimeout) == 0) {
+                    w.status[1] = where;
+                    w.status[2] = static_cast<int>(blockIdx.x);
+                }
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes,
+                                                   uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);         // start address
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;  // leading byte offset
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;  // stride byte offset
+    d |= static_cast<uint64_t>(1) << 46;                         // descriptor version (sm_100)
+    d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
+    return d;
+}
+
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool a_mn, bool b_mn)
+{
+    return (1u << 4)                               // accumulator fp32
+           | (1u << 7) | (1u << 10)                // A, B bf16
+           | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16)
+           | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void decode_unit(const GemmParams &p, int u, int &m_blk, int &n_blk,
+                                            int &split)
+{
+    const int tiles = p.tiles_m * p.tiles_n;
+    split = u / tiles;
+    const int t = u - split * tiles;
+    const int per_group = p.group_m * p.tiles_n;
+    const int g = t / per_group;
+    const int r = t - g * per_group;
+    const int first_m = g * p.group_m;
+    const int gsz = min(p.group_m, p.tiles_m - first_m);
+    m_blk = first_m + r % gsz;
+    n_blk = r / gsz;
+}
+
+__device__ __forceinline__ float gelu_fwd(float z)
+{
+    const float u = 0.7978845608028654f * (z + 0.044715f * z * z * z);
+    return 0.5f * z * (1.0f + ptx::tanh_approx(u));
+}
+__device__ __forceinline__ float gelu_bwd(float x)
+{
+    const float x2 = x * x;
+    const float u = 0.7978845608028654f * (x + 0.044715f * x * x2);
+    const float t = ptx::tanh_approx(u);
+    const float du = 0.7978845608028654f * (1.0f + 3.0f * 0.044715f * x2);
+    return 0.5f * (1.0f + t) + 0.5f * x * (1.0f - t * t) * du;
+}
+__device__ __forceinline__ float silu_fwd(float g) { return __fdividef(g, 1.0f + __expf(-g)); }
+
+template <class Cfg>
+__global__ void __launch_bounds__(kNumThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmE,
+            const GemmParams p)
+{
+    constexpr int BLOCK_N = Cfg::BLOCK_N;
+    constexpr int STAGES = Cfg::STAGES;
+    constexpr int EPI = Cfg::EPI;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t smem = ptx::smem_u32(smem_raw);
+    const int warp = static_cast<int>(threadIdx.x >> 5);
+    const int lane = static_cast<int>(threadIdx.x & 31);
+
+    if ((smem & 1023u) != 0) {  // swizzled tiles need 1024-byte alignment
+        if (threadIdx.x == 0 && atomicCAS(p.status, 0, kStatusBadSmem) == 0)
+            p.status[2] = static_cast<int>(blockIdx.x);
+        return;
+    }
+
+    const uint32_t bar0 = smem + Cfg::OFF_BAR;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+    auto aux_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 4 + b); };
+    const uint32_t tmem_slot = bar0 + 240;
+    const uint32_t abort_addr = bar0 + 244;
+    const uint32_t epi_abort_addr = bar0 + 248;
+    static_assert(8 * (2 * STAGES + 8) <= 240, "barrier region");
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull_bar(b), 1);
+            ptx::mbar_init(tempty_bar(b), 4);
+        }
+        for (int b = 0; b < 4; ++b) ptx::mbar_init(aux_bar(b), 1);
+        ptx::st_shared_u32_volatile(abort_addr, 0);
+        ptx::st_shared_u32_volatile(epi_abort_addr, 0);
+        ptx::fence_barrier_init();
+        ptx::prefetch_tmap(&tmA);
+        ptx::prefetch_tmap(&tmB);
+        ptx::prefetch_tmap(&tmD);
+        if (EPI == kEpiGelu || EPI == kEpiSwiglu || EPI == kEpiMulGeluGrad) ptx::prefetch_tmap(&tmE);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ptx::ld_shared_u32_volatile(tmem_slot);
+
+    const WaitCtx wctx{abort_addr, p.status, p.timeout_ns};
+    const int num_units = p.tiles_m * p.tiles_n * p.splits;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+                int m_blk, n_blk, split;
+                decode_unit(p, u, m_blk, n_blk, split);
+                const int kb0 = split * p.kblocks_per_split;
+                const int kb1 = min(kb0 + p.kblocks_per_split, p.kblocks);
+                const int m0 = m_blk * kBlockM;
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    ok = wait_barrier(wctx, empty_bar(stage), phase ^ 1u, 100 + stage);
+                    if (!ok) break;
+                    const uint32_t fb = full_bar(stage);
+                    ptx::mbar_expect_tx(fb, Cfg::A_BYTES + Cfg::B_BYTES);
+                    const uint32_t sa = smem + Cfg::OFF_A + stage * Cfg::A_BYTES;
+                    const uint32_t sb = smem + Cfg::OFF_B + stage * Cfg::B_BYTES;
+                    const int k0 = kb * kBlockK;
+                    if (Cfg::A_MN) {  // tensor [K rows, M cols]: boxes of 64(m) x 64(k)
+#pragma unroll
+                        for (int j = 0; j < kBlockM / 64; ++j)
+                            ptx::tma_load_2d(sa + j * 8192u, &tmA, fb, m0 + j * 64, k0);
+                    } else {          // tensor [M rows, K cols]: boxes of 64(k) x 64(m)
+#pragma unroll
+                        for (int j = 0; j < kBlockM / 64; ++j)
+                            ptx::tma_load_2d(sa + j * 8192u, &tmA, fb, k0, m0 + j * 64);
+                    }
+                    if (Cfg::B_MN) {
+                        const int n0 = n_blk * BLOCK_N;
+#pragma unroll
+                        for (int j = 0; j < BLOCK_N / 64; ++j)
+                            ptx::tma_load_2d(sb + j * 8192u, &tmB, fb, n0 + j * 64, k0);
+                    } else if (EPI == kEpiSwiglu) {  // 128 gate rows, then the matching 128 up rows
+                        const int n0 = n_blk * 128;
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            ptx::tma_load_2d(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
+                            ptx::tma_load_2d(sb + 16384u + j * 8192u, &tmB, fb, k0,
+                                             p.swiglu_h + n0 + j * 64);
+                        }
+                    } else {                          // boxes of 64(k) x 64(n)
+                        const int n0 = n_blk * BLOCK_N;
+#pragma unroll
+                        for (int j = 0; j < BLOCK_N / 64; ++j)
+                            ptx::tma_load_2d(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
+                    }
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(kBlockM, BLOCK_N, Cfg::A_MN, Cfg::B_MN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+                int m_blk, n_blk, split;
+                decode_unit(p, u, m_blk, n_blk, split);
+                const int kb0 = split * p.kblocks_per_split;
+                const int kb1 = min(kb0 + p.kblocks_per_split, p.kblocks);
+                ok = wait_barrier(wctx, tempty_bar(acc), acc_phase ^ 1u, 200 + acc);
+                if (!ok) break;
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BLOCK_N);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    ok = wait_barrier(wctx, full_bar(stage), phase, 300 + stage);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    const uint32_t sa = smem + Cfg::OFF_A + stage * Cfg::A_BYTES;
+                    const uint32_t sb = smem + Cfg::OFF_B + stage * Cfg::B_BYTES;
+                    // K-major: 8-row groups 1024 B apart, 16 k = 32 B inside the swizzle row.
+                    // MN-major: 64-wide chunks 8192 B apart, 8-k groups 1024 B apart, 16 k = 2048 B.
+                    const uint64_t adesc = Cfg::A_MN ? make_smem_desc(sa, 8192, 1024)
+                                                     : make_smem_desc(sa, 16, 1024);
+                    const uint64_t bdesc = Cfg::B_MN ? make_smem_desc(sb, 8192, 1024)
+                                                     : make_smem_desc(sb, 16, 1024);
+                    constexpr uint32_t a_step = Cfg::A_MN ? (2048u >> 4) : (32u >> 4);
+                    constexpr uint32_t b_step = Cfg::B_MN ? (2048u >> 4) : (32u >> 4);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                        ptx::umma_bf16(d_tmem, adesc + static_cast<uint64_t>(k * a_step),
+                                       bdesc + static_cast<uint64_t>(k * b_step), idesc,
+                                       (kb > kb0 || k > 0) ? 1u : 0u);
+                    }
+                    ptx::umma_commit(empty_bar(stage));  // stage may be refilled once these finish
+                    if (++stage == STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                ptx::umma_commit(tfull_bar(acc));  // accumulator complete
+                if (++acc == 2) {
+                    acc = 0;
+                    acc_phase ^= 1u;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;           // TMEM lane quarter this warp may read
+        const int row = q * 32 + lane;    // row of the tile owned by this thread
+        const bool leader = (threadIdx.x == 64);
+        const int et = static_cast<int>(threadIdx.x) - 64;  // 0..127
+        const uint32_t stg0 = smem + Cfg::OFF_STG;
+        const uint32_t bias_s = smem + Cfg::OFF_BIAS;
+        const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
+        const uint32_t sw = static_cast<uint32_t>(row & 7);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        uint32_t gstep = 0;  // epilogue steps done so far (drives the staging ring)
+        constexpr int SLOTS = Cfg::SLOTS;
+        constexpr int STEPS = Cfg::STEPS;
+        constexpr int AUX_AHEAD = 2;
+
+        // coordinates of the aux tile for global step g (kEpiMulGeluGrad)
+        auto issue_aux = [&](uint32_t g) {
+            const int ui = static_cast<int>(g / STEPS);
+            const int c = static_cast<int>(g % STEPS);
+            const long long u = static_cast<long long>(blockIdx.x) +
+                                static_cast<long long>(ui) * gridDim.x;
+            if (u >= num_units) return;
+            int m_blk, n_blk, split;
+            decode_unit(p, static_cast<int>(u), m_blk, n_blk, split);
+            const int x = n_blk * BLOCK_N + c * 64;
+            const uint32_t slot = g % SLOTS;
+            const uint32_t ab = aux_bar(static_cast<int>(slot));
+            ptx::mbar_expect_tx(ab, kStgBytes);
+            ptx::tma_load_2d(stg0 + slot * kStgBytes, &tmE, ab, x, m_blk * kBlockM);
+        };
+        if (EPI == kEpiMulGeluGrad && leader) {
+            for (uint32_t g = 0; g < AUX_AHEAD; ++g) issue_aux(g);
+        }
+
+        for (int u = blockIdx.x; u < num_units; u += gridDim.x) {
+            // uniform exit: the flag is only written by epilogue threads inside a unit, and
+            // only read here, between the last barrier of one unit and the first of the next
+            if (ptx::ld_shared_u32_volatile(epi_abort_addr) != 0) break;
+            int m_blk, n_blk, split;
+            decode_unit(p, u, m_blk, n_blk, split);
+            const int m0 = m_blk * kBlockM;
+            const int n0 = (EPI == kEpiSwiglu) ? n_blk * 128 : n_blk * BLOCK_N;
+            if (EPI == kEpiStore || EPI == kEpiGelu || EPI == kEpiSwiglu) {
+                for (int i = et; i < BLOCK_N; i += kEpiThreads) {
+                    int col;
+                    if (EPI == kEpiSwiglu) col = (i < 128) ? (n0 + i) : (p.swiglu_h + n0 + i - 128);
+                    else col = n0 + i;
+                    float b = 0.0f;
+                    if (p.bias != nullptr && col < p.N) b = __bfloat162float(p.bias[col]);
+                    ptx::st_shared_f32(bias_s + 4u * i, b);
+                }
+            }
+            ptx::named_bar_sync(1, kEpiThreads);
+
+            bool ok = true;
+            if (lane == 0) ok = wait_barrier(wctx, tfull_bar(acc), acc_phase, 400 + acc);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
+            ptx::tc_fence_after();
+            const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                   static_cast<uint32_t>(acc * BLOCK_N);
+
+#pragma unroll 1
+            for (int c = 0; c < STEPS; ++c, ++gstep) {
+                const uint32_t slot = gstep % SLOTS;
+                const uint32_t buf = stg0 + slot * Cfg::BUFS_PER_STEP * kStgBytes;
+
+                if (EPI == kEpiStore || EPI == kEpiGelu) {
+                    uint32_t r0[32], r1[32];
+                    ptx::tmem_ld_32x32(t_acc + c * 64, r0);
+                    ptx::tmem_ld_32x32(t_acc + c * 64 + 32, r1);
+                    ptx::tmem_ld_wait();
+                    if (c == STEPS - 1) {  // accumulator fully read: hand it back to the MMA warp
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float v[8];
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint32_t bits = (h == 0) ? r0[j * 8 + k] : r1[j * 8 + k];
+                                v[k] = __uint_as_float(bits) +
+                                       ptx::ld_shared_f32(bias_s + 4u * (c * 64 + h * 32 + j * 8 + k));
+                            }
+                            const uint32_t pos = row_off + (((h * 4 + j) ^ sw) << 4);
+                            if (EPI == kEpiGelu) {
+                                ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(v[0], v[1]),
+                                                  ptx::pack_bf16x2(v[2], v[3]),
+                                                  ptx::pack_bf16x2(v[4], v[5]),
+                                                  ptx::pack_bf16x2(v[6], v[7]));
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) v[k] = gelu_fwd(v[k]);
+                            }
+                            ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(v[0], v[1]),
+                                              ptx::pack_bf16x2(v[2], v[3]),
+                                              ptx::pack_bf16x2(v[4], v[5]),
+                                              ptx::pack_bf16x2(v[6], v[7]));
+                        }
+                    }
+                } else if (EPI == kEpiSwiglu) {
+                    // step c covers out columns [c*64, c*64+64): gate TMEM cols c*64.., up cols 128+c*64..
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t rg[32], ru[32];
+                        ptx::tmem_ld_32x32(t_acc + c * 64 + h * 32, rg);
+                        ptx::tmem_ld_32x32(t_acc + 128 + c * 64 + h * 32, ru);
+                        ptx::tmem_ld_wait();
+                        if (c == STEPS - 1 && h == 1) {
+                            ptx::tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            float g[8], uu[8], o[8];
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int cc = c * 64 + h * 32 + j * 8 + k;
+                                g[k] = __uint_as_float(rg[j * 8 + k]) + ptx::ld_shared_f32(bias_s + 4u * cc);
+                                uu[k] = __uint_as_float(ru[j * 8 + k]) +
+                                        ptx::ld_shared_f32(bias_s + 4u * (128 + cc));
+                                o[k] = silu_fwd(g[k]) * uu[k];
+                            }
+                            const uint32_t pos = row_off + (((h * 4 + j) ^ sw) << 4);
+                            ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(o[0], o[1]),
+                                              ptx::pack_bf16x2(o[2], o[3]), ptx::pack_bf16x2(o[4], o[5]),
+                                              ptx::pack_bf16x2(o[6], o[7]));
+                            ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(g[0], g[1]),
+                                              ptx::pack_bf16x2(g[2], g[3]), ptx::pack_bf16x2(g[4], g[5]),
+                                              ptx::pack_bf16x2(g[6], g[7]));
+                            ptx::st_shared_v4(buf + 2 * kStgBytes + pos, ptx::pack_bf16x2(uu[0], uu[1]),
+                                              ptx::pack_bf16x2(uu[2], uu[3]),
+                                              ptx::pack_bf16x2(uu[4], uu[5]),
+                                              ptx::pack_bf16x2(uu[6], uu[7]));
+                        }
+                    }
+                } else if (EPI == kEpiMulGeluGrad) {
+                    bool aok = true;
+                    if (lane == 0)
+                        aok = wait_barrier(wctx, aux_bar(static_cast<int>(slot)), (gstep / SLOTS) & 1u,
+                                           500 + static_cast<int>(slot));
+                    aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
+                    if (!aok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
+                    uint32_t r0[32], r1[32];
+                    ptx::tmem_ld_32x32(t_acc + c * 64, r0);
+                    ptx::tmem_ld_32x32(t_acc + c * 64 + 32, r1);
+                    ptx::tmem_ld_wait();
+                    if (c == STEPS - 1) {
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t pos = buf + row_off + (((h * 4 + j) ^ sw) << 4);
+                            uint32_t x[4];
+                            ptx::ld_shared_v4(pos, x[0], x[1], x[2], x[3]);
+                            uint32_t w[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const uint32_t b0 = (h == 0) ? r0[j * 8 + 2 * k] : r1[j * 8 + 2 * k];
+                                const uint32_t b1 = (h == 0) ? r0[j * 8 + 2 * k + 1] : r1[j * 8 + 2 * k + 1];
+                                const float lo = __uint_as_float(b0) * gelu_bwd(ptx::bf16_lo(x[k]));
+                                const float hi = __uint_as_float(b1) * gelu_bwd(ptx::bf16_hi(x[k]));
+                                w[k] = ptx::pack_bf16x2(lo, hi);
+                            }
+                            ptx::st_shared_v4(pos, w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                } else {  // kEpiF32: 32 fp32 columns per step
+                    uint32_t r0[32];
+                    ptx::tmem_ld_32x32(t_acc + c * 32, r0);
+                    ptx::tmem_ld_wait();
+                    if (c == STEPS - 1) {
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        ptx::st_shared_v4(buf + row_off + ((j ^ sw) << 4), r0[j * 4], r0[j * 4 + 1],
+                                          r0[j * 4 + 2], r0[j * 4 + 3]);
+                }
+
+                // make the staged tile visible to the TMA engine, then one thread stores it
+                ptx::fence_proxy_async_smem();
+                if (leader && SLOTS >= 2) {
+                    // the slot the NEXT step writes was last stored SLOTS-1 groups ago
+                    ptx::bulk_wait_group_read<(SLOTS >= 2 ? SLOTS - 2 : 0)>();
+                }
+                ptx::named_bar_sync(1, kEpiThreads);
+                if (leader) {
+                    if (ok) {
+                        if (EPI == kEpiStore || EPI == kEpiMulGeluGrad) {
+                            const int x = n0 + c * 64;
+                            if (x < p.N) ptx::tma_store_2d(&tmD, buf, x, m0);
+                        } else if (EPI == kEpiGelu) {
+                            const int x = n0 + c * 64;
+                            if (x < p.N) {
+                                ptx::tma_store_2d(&tmD, buf, x, m0);
+                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, m0);
+                            }
+                        } else if (EPI == kEpiSwiglu) {
+                            const int x = n0 + c * 64;
+                            if (x < p.swiglu_h) {
+                                ptx::tma_store_2d(&tmD, buf, x, m0);
+                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, m0);
+                                ptx::tma_store_2d(&tmE, buf + 2 * kStgBytes, p.swiglu_h + x, m0);
+                            }
+                        } else {
+                            const int x = n0 + c * 32;
+                            if (x < p.N) {
+                                if (p.reduce) ptx::tma_reduce_add_2d(&tmD, buf, x, m0);
+                                else ptx::tma_store_2d(&tmD, buf, x, m0);
+                            }
+                        }
+                    }
+                    ptx::bulk_commit_group();
+                    if (EPI == kEpiMulGeluGrad) {
+                        // slot of step gstep+AUX_AHEAD was stored SLOTS-AUX_AHEAD groups ago
+                        ptx::bulk_wait_group_read<(SLOTS > AUX_AHEAD ? SLOTS - AUX_AHEAD : 0)>();
+                        issue_aux(gstep + AUX_AHEAD);
+                    }
+                    if (SLOTS == 1) ptx::bulk_wait_group_read<0>();
+                }
+                if (SLOTS == 1) ptx::named_bar_sync(1, kEpiThreads);
+            }
+            if (++acc == 2) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
+        }
+        if (leader) ptx::bulk_wait_group<0>();  // all stores have reached global memory
+    }
+
+    // ---------------------------------------------------------------- common exit
+    if (ptx::ld_shared_u32_volatile(abort_addr) != 0 ||
+        ptx::ld_shared_u32_volatile(epi_abort_addr) != 0) {
+        // a wait expired somewhere: give copies and MMAs still in flight time to land
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace nb

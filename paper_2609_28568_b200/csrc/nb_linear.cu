@@ -1,0 +1,542 @@
+// Host side of the nb_linear C ABI: argument checks, TMA descriptors, kernel selection, launches.
+// Declarations and argument documentation live in include/nb_linear.h.
+#include "nb_linear.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <unordered_map>
+
+#include "elementwise.cuh"
+#include "gemm_sm100.cuh"
+
+namespace {
+
+using namespace nb;
+
+constexpr int kMaxDevices = 64;
+constexpr unsigned long long kDefaultTimeoutNs = 2000000000ull;  // 2 s per wait
+
+thread_local std::string g_err;
+thread_local cudaStream_t g_stream = nullptr;
+
+int fail(int code, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return code;
+}
+
+#define NB_CUDA(call)                                                                        \
+    do {                                                                                     \
+        cudaError_t e_ = (call);                                                             \
+        if (e_ != cudaSuccess)                                                               \
+            return fail(NB_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));        \
+    } while (0)
+
+// ----------------------------------------------------------------------------- per-device state
+struct TmapKey {
+    const void *ptr;
+    uint64_t rows, cols;
+    uint32_t box_cols, box_rows, dtype;
+    bool operator==(const TmapKey &o) const
+    {
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_cols == o.box_cols &&
+               box_rows == o.box_rows && dtype == o.dtype;
+    }
+};
+struct TmapKeyHash {
+    size_t operator()(const TmapKey &k) const
+    {
+        uint64_t h = reinterpret_cast<uint64_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
+        h ^= (k.rows + 0x7F4A7C15ull) * 0xBF58476D1CE4E5B9ull;
+        h ^= (k.cols + 0x165667B1ull) * 0x94D049BB133111EBull;
+        h ^= (static_cast<uint64_t>(k.box_cols) << 40) ^ (static_cast<uint64_t>(k.box_rows) << 20) ^
+             k.dtype;
+        return static_cast<size_t>(h ^ (h >> 29));
+    }
+};
+
+struct DeviceState {
+    bool init = false;
+    int num_sms = 0;
+    int *status = nullptr;   // 16 ints on the device
+    void *workspace = nullptr;
+    size_t workspace_bytes = 0;
+    std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> tmaps;
+};
+
+std::mutex g_mu;
+DeviceState g_dev[kMaxDevices];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int get_state(DeviceState **out)
+{
+    int dev = 0;
+    NB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(NB_ERR_UNSUPPORTED, "device index %d", dev);
+    DeviceState &s = g_dev[dev];
+    if (!s.init) {
+        cudaDeviceProp prop;
+        NB_CUDA(cudaGetDeviceProperties(&prop, dev));
+        if (prop.major != 10)
+            return fail(NB_ERR_UNSUPPORTED,
+                        "device %d is sm_%d%d; this library only runs on sm_100 (B200)", dev,
+                        prop.major, prop.minor);
+        s.num_sms = prop.multiProcessorCount;
+        NB_CUDA(cudaMalloc(reinterpret_cast<void **>(&s.status), 64));
+        NB_CUDA(cudaMemset(s.status, 0, 64));
+        if (!g_encode) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            NB_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+            if (qres != cudaDriverEntryPointSuccess || !fn)
+                return fail(NB_ERR_CUDA, "cuTensorMapEncodeTiled is not available in this driver");
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        s.init = true;
+    }
+    *out = &s;
+    return NB_OK;
+}
+
+// Row-major [rows, cols] tensor, tiles of box_rows x box_cols with the 128-byte swizzle.
+// dtype: 0 bf16, 1 fp32. The innermost box extent is always 128 bytes (64 bf16 / 32 fp32).
+int get_tmap(DeviceState &s, CUtensorMap *out, const void *ptr, uint64_t rows, uint64_t cols,
+             uint32_t dtype, uint32_t box_rows)
+{
+    const uint32_t esz = dtype == 0 ? 2u : 4u;
+    const uint32_t box_cols = 128u / esz;
+    TmapKey key{ptr, rows, cols, box_cols, box_rows, dtype};
+    auto it = s.tmaps.find(key);
+    if (it != s.tmaps.end()) {
+        *out = it->second;
+        return NB_OK;
+    }
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * esz};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUtensorMap m;
+    CUresult r = g_encode(&m, dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                          2, const_cast<void *>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(NB_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for [%llu, %llu] at %p",
+                    static_cast<int>(r), static_cast<unsigned long long>(rows),
+                    static_cast<unsigned long long>(cols), ptr);
+    if (s.tmaps.size() > 8192) s.tmaps.clear();
+    s.tmaps.emplace(key, m);
+    *out = m;
+    return NB_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_dims(int64_t BT, int64_t C, int64_t OC)
+{
+    if (BT < 0 || C <= 0 || OC <= 0) return fail(NB_ERR_INVALID_ARG, "negative or zero dimension");
+    if (BT >= (1ll << 31) || C >= (1ll << 31) || OC >= (1ll << 31) || BT * OC >= (1ll << 40) ||
+        BT * C >= (1ll << 40))
+        return fail(NB_ERR_UNSUPPORTED, "dimension too large");
+    if (C % 8 != 0 || OC % 8 != 0)
+        return fail(NB_ERR_UNSUPPORTED, "C (%lld) and OC (%lld) must be multiples of 8",
+                    static_cast<long long>(C), static_cast<long long>(OC));
+    return NB_OK;
+}
+
+// ----------------------------------------------------------------------------- GEMM launch
+struct GemmArgs {
+    const void *A;  uint64_t a_rows, a_cols;   // global tensor of the A operand (bf16)
+    const void *B;  uint64_t b_rows, b_cols;   // global tensor of the B operand (bf16)
+    void *D;        uint64_t d_rows, d_cols;  uint32_t d_dtype;
+    const void *E;  uint64_t e_rows, e_cols;   // second bf16 tensor (pre-activation / aux) or null
+    int M, N, K;
+    const void *bias;
+    int swiglu_h;
+    int reduce;
+    int splits;
+};
+
+template <class Cfg>
+int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
+{
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    NB_CUDA(cudaGetDevice(&dev));
+    if (!attr_set[dev]) {
+        NB_CUDA(cudaFuncSetAttribute(gemm_kernel<Cfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(Cfg::SMEM_BYTES)));
+        attr_set[dev] = true;
+    }
+    CUtensorMap tA, tB, tD, tE;
+    int rc;
+    // operands are fetched as 64 x 64 boxes; results (and the aux tile) move as 128-row chunks
+    if ((rc = get_tmap(s, &tA, a.A, a.a_rows, a.a_cols, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tB, a.B, a.b_rows, a.b_cols, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tD, a.D, a.d_rows, a.d_cols, a.d_dtype, kBlockM)) != NB_OK) return rc;
+    if (a.E) {
+        if ((rc = get_tmap(s, &tE, a.E, a.e_rows, a.e_cols, 0, kBlockM)) != NB_OK) return rc;
+    } else {
+        tE = tD;
+    }
+    GemmParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = a.M;
+    p.N = a.N;
+    p.K = a.K;
+    p.tiles_m = (a.M + kBlockM - 1) / kBlockM;
+    const int n_span = (Cfg::EPI == kEpiSwiglu) ? a.swiglu_h : a.N;
+    const int n_tile = (Cfg::EPI == kEpiSwiglu) ? 128 : Cfg::BLOCK_N;
+    p.tiles_n = (n_span + n_tile - 1) / n_tile;
+    p.kblocks = (a.K + kBlockK - 1) / kBlockK;
+    int splits = a.splits < 1 ? 1 : a.splits;
+    if (splits > p.kblocks) splits = p.kblocks;
+    p.kblocks_per_split = (p.kblocks + splits - 1) / splits;
+    p.splits = (p.kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;
+    p.group_m = 16;
+    p.swiglu_h = a.swiglu_h;
+    p.reduce = a.reduce;
+    p.bias = static_cast<const __nv_bfloat16 *>(a.bias);
+    p.status = s.status;
+    p.timeout_ns = kDefaultTimeoutNs;
+    const long long units = 1ll * p.tiles_m * p.tiles_n * p.splits;
+    if (units <= 0 || units >= (1ll << 31)) return fail(NB_ERR_UNSUPPORTED, "tile count out of range");
+    const int grid = static_cast<int>(units < s.num_sms ? units : s.num_sms);
+    gemm_kernel<Cfg><<<grid, kNumThreads, Cfg::SMEM_BYTES, stream>>>(tA, tB, tD, tE, p);
+    NB_CUDA(cudaGetLastError());
+    return NB_OK;
+}
+
+// kernel configurations: <BLOCK_N, STAGES, staging buffers, A MN-major, B MN-major, epilogue>
+using FwdStore = GemmCfg<256, 4, 2, false, false, kEpiStore>;
+using FwdGelu = GemmCfg<256, 3, 4, false, false, kEpiGelu>;
+using FwdSwiglu = GemmCfg<256, 3, 3, false, false, kEpiSwiglu>;
+using DgradStore = GemmCfg<256, 4, 2, false, true, kEpiStore>;
+using DgradMulGelu = GemmCfg<256, 3, 4, false, true, kEpiMulGeluGrad>;
+using WgradF32 = GemmCfg<256, 4, 2, true, true, kEpiF32>;
+using WgradBf16 = GemmCfg<256, 4, 2, true, true, kEpiStore>;
+
+int ensure_workspace(DeviceState &s, size_t bytes)
+{
+    if (s.workspace_bytes >= bytes) return NB_OK;
+    if (s.workspace) {
+        NB_CUDA(cudaDeviceSynchronize());
+        NB_CUDA(cudaFree(s.workspace));
+        s.workspace = nullptr;
+        s.workspace_bytes = 0;
+    }
+    const size_t want = (bytes + (1u << 20) - 1) & ~static_cast<size_t>((1u << 20) - 1);
+    NB_CUDA(cudaMalloc(&s.workspace, want));
+    s.workspace_bytes = want;
+    return NB_OK;
+}
+
+int launch_dbias(DeviceState &s, float *dbias, const void *dz, int64_t BT, int64_t OC, int accumulate,
+                 cudaStream_t stream)
+{
+    if (!accumulate) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
+    if (BT == 0) return NB_OK;
+    const int col_blocks = static_cast<int>((OC + kDbiasCols - 1) / kDbiasCols);
+    long long want_row_blocks = (8ll * s.num_sms + col_blocks - 1) / col_blocks;
+    long long rows_per_block = (BT + want_row_blocks - 1) / want_row_blocks;
+    rows_per_block = ((rows_per_block + 31) / 32) * 32;
+    if (rows_per_block < 32) rows_per_block = 32;
+    const long long row_blocks = (BT + rows_per_block - 1) / rows_per_block;
+    if (row_blocks > 65535) return fail(NB_ERR_UNSUPPORTED, "BT too large for the dbias grid");
+    dim3 grid(col_blocks, static_cast<unsigned>(row_blocks));
+    dbias_kernel<<<grid, kDbiasThreads, 0, stream>>>(dbias, static_cast<const __nv_bfloat16 *>(dz), BT,
+                                                     static_cast<int>(OC),
+                                                     static_cast<int>(rows_per_block));
+    NB_CUDA(cudaGetLastError());
+    return NB_OK;
+}
+
+int elementwise_grid(const DeviceState &s, long long nvec)
+{
+    long long blocks = (nvec + 255) / 256;
+    const long long cap = 16ll * s.num_sms;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return static_cast<int>(blocks);
+}
+
+}  // namespace
+
+// ================================================================================ C ABI
+extern "C" {
+
+int nb_version(void) { return 100; }
+
+const char *nb_last_error(void) { return g_err.c_str(); }
+
+int nb_set_stream(void *stream)
+{
+    g_stream = static_cast<cudaStream_t>(stream);
+    return NB_OK;
+}
+void *nb_get_stream(void) { return g_stream; }
+
+int64_t nb_linear_out_elems(int64_t BT, int64_t OC, int act)
+{
+    if (BT < 0 || OC < 0) return -1;
+    switch (act) {
+        case NB_ACT_NONE: return BT * OC;
+        case NB_ACT_GELU: return 2 * BT * OC;
+        case NB_ACT_SWIGLU: return (OC % 2) ? -1 : BT * (OC / 2) + BT * OC;
+        default: return -1;
+    }
+}
+
+int nb_linear_forward_ex(void *out, void *pre_act, const void *inp, const void *weight,
+                         const void *bias, int64_t BT, int64_t C, int64_t OC, int act, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (act != NB_ACT_NONE && act != NB_ACT_GELU && act != NB_ACT_SWIGLU)
+        return fail(NB_ERR_INVALID_ARG, "unknown activation %d", act);
+    int rc = check_dims(BT, C, OC);
+    if (rc != NB_OK) return rc;
+    if (act == NB_ACT_SWIGLU && OC % 16 != 0)
+        return fail(NB_ERR_UNSUPPORTED, "SwiGLU needs OC/2 to be a multiple of 8");
+    if (!out || !inp || !weight) return fail(NB_ERR_INVALID_ARG, "out, inp and weight must not be NULL");
+    if (!aligned16(out) || !aligned16(inp) || !aligned16(weight) || !aligned16(pre_act) ||
+        (bias && (reinterpret_cast<uintptr_t>(bias) & 1u)))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (BT == 0) return NB_OK;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = weight; a.b_rows = OC; a.b_cols = C;
+    a.D = out; a.d_rows = BT; a.d_cols = (act == NB_ACT_SWIGLU) ? OC / 2 : OC; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(OC); a.K = static_cast<int>(C);
+    a.bias = bias;
+    a.splits = 1;
+    if (act == NB_ACT_NONE) return launch_gemm<FwdStore>(*s, a, stream);
+    if (!pre_act) {
+        // the activated result without its pre-activation: only NONE can skip the second plane
+        return fail(NB_ERR_INVALID_ARG, "pre_act must be given when act != NONE");
+    }
+    a.E = pre_act; a.e_rows = BT; a.e_cols = OC;
+    if (act == NB_ACT_GELU) return launch_gemm<FwdGelu>(*s, a, stream);
+    a.swiglu_h = static_cast<int>(OC / 2);
+    return launch_gemm<FwdSwiglu>(*s, a, stream);
+}
+
+int nb_linear_forward(void *out, const void *inp, const void *weight, const void *bias, int64_t BT,
+                      int64_t C, int64_t OC, int act)
+{
+    void *pre = nullptr;
+    if (out && BT >= 0 && OC >= 0) {
+        if (act == NB_ACT_GELU) pre = static_cast<uint16_t *>(out) + BT * OC;
+        if (act == NB_ACT_SWIGLU) pre = static_cast<uint16_t *>(out) + BT * (OC / 2);
+    }
+    return nb_linear_forward_ex(out, pre, inp, weight, bias, BT, C, OC, act, g_stream);
+}
+
+int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *dout, const void *inp,
+                          const void *weight, const void *pre_act, const void *inp_pre_act,
+                          int64_t BT, int64_t C, int64_t OC, int act, int accumulate,
+                          int dweight_dtype, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (act != NB_ACT_NONE && act != NB_ACT_GELU && act != NB_ACT_SWIGLU)
+        return fail(NB_ERR_INVALID_ARG, "unknown activation %d", act);
+    if (dweight_dtype != NB_DTYPE_F32 && dweight_dtype != NB_DTYPE_BF16)
+        return fail(NB_ERR_INVALID_ARG, "unknown dweight dtype %d", dweight_dtype);
+    int rc = check_dims(BT, C, OC);
+    if (rc != NB_OK) return rc;
+    if (act == NB_ACT_SWIGLU && OC % 16 != 0)
+        return fail(NB_ERR_UNSUPPORTED, "SwiGLU needs OC/2 to be a multiple of 8");
+    if (!dout) return fail(NB_ERR_INVALID_ARG, "dout must not be NULL");
+    if (act != NB_ACT_NONE && !pre_act)
+        return fail(NB_ERR_INVALID_ARG, "pre_act is required when act != NONE");
+    if (dinp && !weight) return fail(NB_ERR_INVALID_ARG, "weight is required to compute dinp");
+    if (dweight && !inp) return fail(NB_ERR_INVALID_ARG, "inp is required to compute dweight");
+    if (inp_pre_act && !dinp) return fail(NB_ERR_INVALID_ARG, "inp_pre_act given without dinp");
+    if (dweight_dtype == NB_DTYPE_BF16 && accumulate && dweight)
+        return fail(NB_ERR_UNSUPPORTED, "bf16 dweight cannot be accumulated across micro-steps");
+    if (!aligned16(dinp) || !aligned16(dweight) || !aligned16(dbias) || !aligned16(dout) ||
+        !aligned16(inp) || !aligned16(weight) || !aligned16(pre_act) || !aligned16(inp_pre_act))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+
+    if (BT == 0) {
+        if (!accumulate) {
+            const size_t wsz = dweight_dtype == NB_DTYPE_F32 ? 4 : 2;
+            if (dweight) NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(OC * C) * wsz, stream));
+            if (dbias) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
+        }
+        return NB_OK;
+    }
+
+    // dz: either dout itself, or dout times this layer's activation derivative (workspace)
+    const void *dz = dout;
+    if (act != NB_ACT_NONE) {
+        if ((rc = ensure_workspace(*s, static_cast<size_t>(BT * OC) * 2)) != NB_OK) return rc;
+        if (act == NB_ACT_GELU) {
+            const long long nvec = BT * OC / 8;
+            gelu_backward_kernel<<<elementwise_grid(*s, nvec), 256, 0, stream>>>(
+                static_cast<uint4 *>(s->workspace), static_cast<const uint4 *>(dout),
+                static_cast<const uint4 *>(pre_act), nvec);
+        } else {
+            const int hvec = static_cast<int>(OC / 16);
+            swiglu_backward_kernel<<<elementwise_grid(*s, BT * hvec), 256, 0, stream>>>(
+                static_cast<uint4 *>(s->workspace), static_cast<const uint4 *>(dout),
+                static_cast<const uint4 *>(pre_act), BT, hvec);
+        }
+        NB_CUDA(cudaGetLastError());
+        dz = s->workspace;
+    }
+
+    if (dinp) {  // dinp[BT, C] = dz[BT, OC] . W[OC, C]
+        GemmArgs a;
+        memset(&a, 0, sizeof(a));
+        a.A = dz; a.a_rows = BT; a.a_cols = OC;
+        a.B = weight; a.b_rows = OC; a.b_cols = C;
+        a.D = dinp; a.d_rows = BT; a.d_cols = C; a.d_dtype = 0;
+        a.M = static_cast<int>(BT); a.N = static_cast<int>(C); a.K = static_cast<int>(OC);
+        a.splits = 1;
+        if (inp_pre_act) {
+            a.E = inp_pre_act; a.e_rows = BT; a.e_cols = C;
+            rc = launch_gemm<DgradMulGelu>(*s, a, stream);
+        } else {
+            rc = launch_gemm<DgradStore>(*s, a, stream);
+        }
+        if (rc != NB_OK) return rc;
+    }
+
+    if (dweight) {  // dweight[OC, C] (+)= dz^T[OC, BT] . inp[BT, C]
+        GemmArgs a;
+        memset(&a, 0, sizeof(a));
+        a.A = dz; a.a_rows = BT; a.a_cols = OC;
+        a.B = inp; a.b_rows = BT; a.b_cols = C;
+        a.D = dweight; a.d_rows = OC; a.d_cols = C;
+        a.M = static_cast<int>(OC); a.N = static_cast<int>(C); a.K = static_cast<int>(BT);
+        if (dweight_dtype == NB_DTYPE_F32) {
+            a.d_dtype = 1;
+            const int tiles = ((a.M + kBlockM - 1) / kBlockM) * ((a.N + 255) / 256);
+            const int kblocks = (a.K + kBlockK - 1) / kBlockK;
+            int splits = (2 * s->num_sms + tiles - 1) / tiles;
+            if (splits > kblocks / 4) splits = kblocks / 4;
+            if (splits < 1) splits = 1;
+            a.splits = splits;
+            a.reduce = (accumulate || splits > 1) ? 1 : 0;
+            if (!accumulate && splits > 1)
+                NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(OC * C) * 4, stream));
+            rc = launch_gemm<WgradF32>(*s, a, stream);
+        } else {
+            a.d_dtype = 0;
+            a.splits = 1;
+            rc = launch_gemm<WgradBf16>(*s, a, stream);
+        }
+        if (rc != NB_OK) return rc;
+    }
+
+    if (dbias) {
+        if ((rc = launch_dbias(*s, static_cast<float *>(dbias), dz, BT, OC, accumulate, stream)) != NB_OK)
+            return rc;
+    }
+    return NB_OK;
+}
+
+int nb_linear_backward(void *dinp, void *dweight, void *dbias, const void *dout, const void *inp,
+                       const void *weight, const void *pre_act, int64_t BT, int64_t C, int64_t OC,
+                       int accumulate)
+{
+    return nb_linear_backward_ex(dinp, dweight, dbias, dout, inp, weight, pre_act, nullptr, BT, C, OC,
+                                 pre_act ? NB_ACT_GELU : NB_ACT_NONE, accumulate, NB_DTYPE_F32,
+                                 g_stream);
+}
+
+int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int accumulate)
+{
+    if (!dbias || !dout) return fail(NB_ERR_INVALID_ARG, "dbias and dout must not be NULL");
+    if (BT < 0 || OC <= 0) return fail(NB_ERR_INVALID_ARG, "negative or zero dimension");
+    if (OC % 8 != 0) return fail(NB_ERR_UNSUPPORTED, "OC must be a multiple of 8");
+    if (!aligned16(dbias) || !aligned16(dout))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    return launch_dbias(*s, static_cast<float *>(dbias), dout, BT, OC, accumulate, g_stream);
+}
+
+int nb_workspace_reserve(int64_t bytes)
+{
+    if (bytes < 0) return fail(NB_ERR_INVALID_ARG, "negative size");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    return ensure_workspace(*s, static_cast<size_t>(bytes));
+}
+
+int nb_release(void)
+{
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    NB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(NB_ERR_UNSUPPORTED, "device index %d", dev);
+    DeviceState &s = g_dev[dev];
+    if (!s.init) return NB_OK;
+    NB_CUDA(cudaDeviceSynchronize());
+    if (s.workspace) NB_CUDA(cudaFree(s.workspace));
+    if (s.status) NB_CUDA(cudaFree(s.status));
+    s = DeviceState();
+    return NB_OK;
+}
+
+int nb_check_status(void)
+{
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    NB_CUDA(cudaDeviceSynchronize());
+    int host[4] = {0, 0, 0, 0};
+    NB_CUDA(cudaMemcpy(host, s->status, sizeof(host), cudaMemcpyDeviceToHost));
+    if (host[0] == 0) return NB_OK;
+    NB_CUDA(cudaMemset(s->status, 0, 64));
+    if (host[0] == kStatusTimeout)
+        return fail(NB_ERR_TIMEOUT, "a bounded device wait expired (wait id %d, block %d)", host[1],
+                    host[2]);
+    return fail(NB_ERR_CUDA, "kernel reported internal error %d (block %d)", host[0], host[2]);
+}
+
+int nb_debug_wait_timeout(int64_t limit_us)
+{
+    if (limit_us < 1 || limit_us > 1000000)
+        return fail(NB_ERR_INVALID_ARG, "limit_us must be within [1, 1000000]");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    wait_timeout_kernel<<<1, 32, 0, g_stream>>>(s->status, static_cast<unsigned long long>(limit_us) * 1000ull);
+    NB_CUDA(cudaGetLastError());
+    return NB_OK;
+}
+
+}  // extern "C"

@@ -89,8 +89,8 @@ int nb_linear_forward(void *out, const void *inp, const void *weight, const void
 
 /*
  * Forward with the pre-activation plane and the stream given explicitly.
- * pre_act: [BT, OC] bf16, written when act != NONE (may be NULL to skip storing it;
- * must be NULL or ignored for act == NONE). nb_linear_forward wraps this call.
+ * pre_act: [BT, OC] bf16, required and written when act != NONE, ignored for
+ * act == NONE. nb_linear_forward wraps this call.
  */
 int nb_linear_forward_ex(void *out, void *pre_act, const void *inp, const void *weight,
                          const void *bias, int64_t BT, int64_t C, int64_t OC, int act,
@@ -164,6 +164,12 @@ int nb_release(void);
  * pending (NB_ERR_CUDA). Clears the device status word.
  */
 int nb_check_status(void);
+
+/*
+ * Number of kernels this library has launched from the calling process since it was
+ * loaded (memsets issued through the CUDA runtime are not counted).
+ */
+int64_t nb_kernel_launches(void);
 
 /*
  * Self-test of the bounded-wait mechanism: launches a one-block kernel that waits, for

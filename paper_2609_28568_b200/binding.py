@@ -22,7 +22,7 @@ EXPORTS = (
     "nb_version", "nb_last_error", "nb_set_stream", "nb_get_stream", "nb_linear_out_elems",
     "nb_linear_forward", "nb_linear_forward_ex", "nb_linear_backward", "nb_linear_backward_ex",
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
-    "nb_debug_wait_timeout",
+    "nb_debug_wait_timeout", "nb_kernel_launches",
 )
 
 _lib = None
@@ -57,6 +57,7 @@ def lib() -> ctypes.CDLL:
         L.nb_reduce_dbias.argtypes = [_vp, _vp, _i64, _i64, _int]
         L.nb_workspace_reserve.argtypes = [_i64]
         L.nb_debug_wait_timeout.argtypes = [_i64]
+        L.nb_kernel_launches.restype = _i64
         _lib = L
     return _lib
 
@@ -136,6 +137,10 @@ def nb_release() -> None:
 def nb_check_status() -> None:
     """Synchronise and raise NbError(NB_ERR_TIMEOUT / NB_ERR_CUDA) if a kernel reported a failure."""
     _check(lib().nb_check_status())
+
+
+def nb_kernel_launches() -> int:
+    return int(lib().nb_kernel_launches())
 
 
 def nb_debug_wait_timeout(limit_us: int) -> None:

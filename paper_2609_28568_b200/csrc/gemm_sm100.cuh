@@ -12,6 +12,13 @@
 // are fetched as 64(k) x 64(mn) boxes and described to the tensor core as MN-major, so no
 // transpose is ever materialised.
 //
+// CTA pairs (CG = 2). Two CTAs of a cluster share one 256-row tile: each loads its own 128 rows of
+// A and its own half of B's N extent, the leader CTA issues tcgen05.mma.cta_group::2 reading both
+// CTAs' shared memory, and each CTA's TMEM receives its 128 rows of the result. Per SM this halves
+// the B traffic and the stage size, which buys a deeper ring. Both CTAs' loads are counted on the
+// leader's "full" barrier; MMA completion is multicast to both CTAs' "empty" / "tmem_full" barriers;
+// both CTAs' epilogues arrive on the leader's "tmem_empty" barrier.
+//
 // Every wait on an mbarrier is bounded in time; on expiry the kernel records the event in the
 // status word, stops issuing work, and all threads leave through the common exit.
 #pragma once
@@ -50,8 +57,10 @@ struct GemmParams {
     unsigned long long timeout_ns;
 };
 
-template <int BLOCK_N_, int STAGES_, int NSTG_, bool A_MN_, bool B_MN_, int EPI_>
+template <int CG_, int BLOCK_N_, int STAGES_, int NSTG_, bool A_MN_, bool B_MN_, int EPI_>
 struct GemmCfg {
+    static constexpr int CG = CG_;              // CTAs per tile: 1, or 2 (a cta_group::2 pair)
+    static constexpr int TILE_M = kBlockM * CG_;
     static constexpr int BLOCK_N = BLOCK_N_;
     static constexpr int STAGES = STAGES_;
     static constexpr int NSTG = NSTG_;
@@ -59,7 +68,8 @@ struct GemmCfg {
     static constexpr bool B_MN = B_MN_;
     static constexpr int EPI = EPI_;
     static constexpr uint32_t A_BYTES = kBlockM * kBlockK * 2;
-    static constexpr uint32_t B_BYTES = BLOCK_N * kBlockK * 2;
+    static constexpr int B_ROWS = BLOCK_N / CG_;  // rows of B's N extent held by one CTA
+    static constexpr uint32_t B_BYTES = B_ROWS * kBlockK * 2;
     static constexpr uint32_t OFF_A = 0;
     static constexpr uint32_t OFF_B = STAGES * A_BYTES;
     static constexpr uint32_t OFF_STG = STAGES * (A_BYTES + B_BYTES);
@@ -75,7 +85,8 @@ struct GemmCfg {
     static constexpr int SLOTS = NSTG / BUFS_PER_STEP;
     static constexpr int STEPS = (EPI == kEpiF32) ? BLOCK_N / 32
                                  : (EPI == kEpiSwiglu) ? BLOCK_N / 128 : BLOCK_N / 64;
-    static_assert(BLOCK_N % 64 == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
+    static_assert(CG_ == 1 || CG_ == 2, "CTAs per tile");
+    static_assert(BLOCK_N % (64 * CG_) == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
     static_assert(2 * BLOCK_N <= 512, "two accumulators must fit in TMEM");
     static_assert(NSTG % BUFS_PER_STEP == 0 && SLOTS >= 1, "staging ring");
     static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 3, "aux prefetch needs a ring of >= 3");
@@ -178,16 +189,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     constexpr int BLOCK_N = Cfg::BLOCK_N;
     constexpr int STAGES = Cfg::STAGES;
     constexpr int EPI = Cfg::EPI;
+    constexpr int CG = Cfg::CG;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem = ptx::smem_u32(smem_raw);
     const int warp = static_cast<int>(threadIdx.x >> 5);
     const int lane = static_cast<int>(threadIdx.x & 31);
+    // position in the CTA pair; pairs are consecutive blocks along x, so this equals %cluster_ctarank
+    // (taken from blockIdx so the compiler can see that it is uniform across the block)
+    const uint32_t rank = (CG == 2) ? (blockIdx.x & 1u) : 0u;
+    const int first_unit = static_cast<int>(blockIdx.x) / CG;       // units are shared by the pair
+    const int unit_stride = static_cast<int>(gridDim.x) / CG;
 
-    if ((smem & 1023u) != 0) {  // swizzled tiles need 1024-byte alignment
-        if (threadIdx.x == 0 && atomicCAS(p.status, 0, kStatusBadSmem) == 0)
-            p.status[2] = static_cast<int>(blockIdx.x);
-        return;
-    }
+    // swizzled tiles need 1024-byte alignment; if the base is off, record it and do no work
+    const bool smem_ok = (smem & 1023u) == 0;
+    if (!smem_ok && threadIdx.x == 0 && atomicCAS(p.status, 0, kStatusBadSmem) == 0)
+        p.status[2] = static_cast<int>(blockIdx.x);
 
     const uint32_t bar0 = smem + Cfg::OFF_BAR;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -207,7 +223,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 4);
+            ptx::mbar_init(tempty_bar(b), 4 * CG);  // one arrive per epilogue warp of the tile
         }
         for (int b = 0; b < 4; ++b) ptx::mbar_init(aux_bar(b), 1);
         ptx::st_shared_u32_volatile(abort_addr, 0);
@@ -219,64 +235,77 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (EPI == kEpiGelu || EPI == kEpiSwiglu || EPI == kEpiMulGeluGrad) ptx::prefetch_tmap(&tmE);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
-        ptx::tmem_relinquish();
+        ptx::tmem_alloc<CG>(tmem_slot, Cfg::TMEM_COLS);
+        ptx::tmem_relinquish<CG>();
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CG == 2) ptx::cluster_sync();  // the peer's barriers are initialised before anyone signals them
+    else __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = ptx::ld_shared_u32_volatile(tmem_slot);
 
     const WaitCtx wctx{abort_addr, p.status, p.timeout_ns};
     const int num_units = p.tiles_m * p.tiles_n * p.splits;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+    // one tile load, counted on the leader CTA's barrier
+    auto load = [&](uint32_t dst, const CUtensorMap *m, uint32_t bar, int x, int y) {
+        if (CG == 2) ptx::tma_load_2d_pair(dst, m, bar, x, y);
+        else ptx::tma_load_2d(dst, m, bar, x, y);
+    };
+
+    if (!smem_ok) {
+        // fall through to the common exit
+    } else if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (every CTA)
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+            for (int u = first_unit; u < num_units && ok; u += unit_stride) {
                 int m_blk, n_blk, split;
                 decode_unit(p, u, m_blk, n_blk, split);
                 const int kb0 = split * p.kblocks_per_split;
                 const int kb1 = min(kb0 + p.kblocks_per_split, p.kblocks);
-                const int m0 = m_blk * kBlockM;
+                const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     ok = wait_barrier(wctx, empty_bar(stage), phase ^ 1u, 100 + stage);
                     if (!ok) break;
-                    const uint32_t fb = full_bar(stage);
-                    ptx::mbar_expect_tx(fb, Cfg::A_BYTES + Cfg::B_BYTES);
+                    // the leader's barrier collects the bytes of both CTAs of a pair
+                    const uint32_t fb = (CG == 2) ? ptx::mapa(full_bar(stage), 0) : full_bar(stage);
+                    if (rank == 0) ptx::mbar_expect_tx(full_bar(stage), CG * (Cfg::A_BYTES + Cfg::B_BYTES));
                     const uint32_t sa = smem + Cfg::OFF_A + stage * Cfg::A_BYTES;
                     const uint32_t sb = smem + Cfg::OFF_B + stage * Cfg::B_BYTES;
                     const int k0 = kb * kBlockK;
                     if (Cfg::A_MN) {  // tensor [K rows, M cols]: boxes of 64(m) x 64(k)
 #pragma unroll
                         for (int j = 0; j < kBlockM / 64; ++j)
-                            ptx::tma_load_2d(sa + j * 8192u, &tmA, fb, m0 + j * 64, k0);
+                            load(sa + j * 8192u, &tmA, fb, m0 + j * 64, k0);
                     } else {          // tensor [M rows, K cols]: boxes of 64(k) x 64(m)
 #pragma unroll
                         for (int j = 0; j < kBlockM / 64; ++j)
-                            ptx::tma_load_2d(sa + j * 8192u, &tmA, fb, k0, m0 + j * 64);
+                            load(sa + j * 8192u, &tmA, fb, k0, m0 + j * 64);
                     }
+                    // this CTA's share of B's N extent: all of it, or its half of the pair's tile
                     if (Cfg::B_MN) {
-                        const int n0 = n_blk * BLOCK_N;
+                        const int n0 = n_blk * BLOCK_N + static_cast<int>(rank) * Cfg::B_ROWS;
 #pragma unroll
-                        for (int j = 0; j < BLOCK_N / 64; ++j)
-                            ptx::tma_load_2d(sb + j * 8192u, &tmB, fb, n0 + j * 64, k0);
+                        for (int j = 0; j < Cfg::B_ROWS / 64; ++j)
+                            load(sb + j * 8192u, &tmB, fb, n0 + j * 64, k0);
                     } else if (EPI == kEpiSwiglu) {  // 128 gate rows, then the matching 128 up rows
                         const int n0 = n_blk * 128;
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
-                            ptx::tma_load_2d(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
-                            ptx::tma_load_2d(sb + 16384u + j * 8192u, &tmB, fb, k0,
-                                             p.swiglu_h + n0 + j * 64);
+                            if (CG == 1 || rank == 0)
+                                load(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
+                            if (CG == 1 || rank == 1)
+                                load(sb + (CG == 1 ? 16384u : 0u) + j * 8192u, &tmB, fb, k0,
+                                     p.swiglu_h + n0 + j * 64);
                         }
                     } else {                          // boxes of 64(k) x 64(n)
-                        const int n0 = n_blk * BLOCK_N;
+                        const int n0 = n_blk * BLOCK_N + static_cast<int>(rank) * Cfg::B_ROWS;
 #pragma unroll
-                        for (int j = 0; j < BLOCK_N / 64; ++j)
-                            ptx::tma_load_2d(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
+                        for (int j = 0; j < Cfg::B_ROWS / 64; ++j)
+                            load(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
                     }
                     if (++stage == STAGES) {
                         stage = 0;
@@ -286,15 +315,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(kBlockM, BLOCK_N, Cfg::A_MN, Cfg::B_MN);
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc(Cfg::TILE_M, BLOCK_N, Cfg::A_MN, Cfg::B_MN);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < num_units && ok; u += gridDim.x) {
+            for (int u = first_unit; u < num_units && ok; u += unit_stride) {
                 int m_blk, n_blk, split;
                 decode_unit(p, u, m_blk, n_blk, split);
                 const int kb0 = split * p.kblocks_per_split;
@@ -319,18 +348,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     constexpr uint32_t b_step = Cfg::B_MN ? (2048u >> 4) : (32u >> 4);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        ptx::umma_bf16(d_tmem, adesc + static_cast<uint64_t>(k * a_step),
+                        ptx::umma_bf16<CG>(d_tmem, adesc + static_cast<uint64_t>(k * a_step),
                                        bdesc + static_cast<uint64_t>(k * b_step), idesc,
                                        (kb > kb0 || k > 0) ? 1u : 0u);
                     }
-                    ptx::umma_commit(empty_bar(stage));  // stage may be refilled once these finish
+                    ptx::umma_commit<CG>(empty_bar(stage));  // stage may be refilled once these finish
                     if (++stage == STAGES) {
                         stage = 0;
                         phase ^= 1u;
                     }
                 }
                 if (!ok) break;
-                ptx::umma_commit(tfull_bar(acc));  // accumulator complete
+                ptx::umma_commit<CG>(tfull_bar(acc));  // accumulator complete
                 if (++acc == 2) {
                     acc = 0;
                     acc_phase ^= 1u;
@@ -358,8 +387,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         auto issue_aux = [&](uint32_t g) {
             const int ui = static_cast<int>(g / STEPS);
             const int c = static_cast<int>(g % STEPS);
-            const long long u = static_cast<long long>(blockIdx.x) +
-                                static_cast<long long>(ui) * gridDim.x;
+            const long long u = static_cast<long long>(first_unit) +
+                                static_cast<long long>(ui) * unit_stride;
             if (u >= num_units) return;
             int m_blk, n_blk, split;
             decode_unit(p, static_cast<int>(u), m_blk, n_blk, split);
@@ -367,19 +396,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t slot = g % SLOTS;
             const uint32_t ab = aux_bar(static_cast<int>(slot));
             ptx::mbar_expect_tx(ab, kStgBytes);
-            ptx::tma_load_2d(stg0 + slot * kStgBytes, &tmE, ab, x, m_blk * kBlockM);
+            ptx::tma_load_2d(stg0 + slot * kStgBytes, &tmE, ab, x,
+                             m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM);
         };
         if (EPI == kEpiMulGeluGrad && leader) {
             for (uint32_t g = 0; g < AUX_AHEAD; ++g) issue_aux(g);
         }
 
-        for (int u = blockIdx.x; u < num_units; u += gridDim.x) {
+        // the accumulator is handed back on the leader CTA's barrier
+        auto release_acc = [&](int a) {
+            if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(a), 0));
+            else ptx::mbar_arrive(tempty_bar(a));
+        };
+
+        for (int u = first_unit; u < num_units; u += unit_stride) {
             // uniform exit: the flag is only written by epilogue threads inside a unit, and
             // only read here, between the last barrier of one unit and the first of the next
             if (ptx::ld_shared_u32_volatile(epi_abort_addr) != 0) break;
             int m_blk, n_blk, split;
             decode_unit(p, u, m_blk, n_blk, split);
-            const int m0 = m_blk * kBlockM;
+            const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
             const int n0 = (EPI == kEpiSwiglu) ? n_blk * 128 : n_blk * BLOCK_N;
             if (EPI == kEpiStore || EPI == kEpiGelu || EPI == kEpiSwiglu) {
                 for (int i = et; i < BLOCK_N; i += kEpiThreads) {
@@ -408,13 +444,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
                 if (EPI == kEpiStore || EPI == kEpiGelu) {
                     uint32_t r0[32], r1[32];
-                    ptx::tmem_ld_32x32(t_acc + c * 64, r0);
-                    ptx::tmem_ld_32x32(t_acc + c * 64 + 32, r1);
-                    ptx::tmem_ld_wait();
+                    ptx::tmem_ld_32x32_x2_wait(t_acc + c * 64, t_acc + c * 64 + 32, r0, r1);
                     if (c == STEPS - 1) {  // accumulator fully read: hand it back to the MMA warp
                         ptx::tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                        if (lane == 0) release_acc(acc);
                     }
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
@@ -447,13 +481,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         uint32_t rg[32], ru[32];
-                        ptx::tmem_ld_32x32(t_acc + c * 64 + h * 32, rg);
-                        ptx::tmem_ld_32x32(t_acc + 128 + c * 64 + h * 32, ru);
-                        ptx::tmem_ld_wait();
+                        ptx::tmem_ld_32x32_x2_wait(t_acc + c * 64 + h * 32, t_acc + 128 + c * 64 + h * 32,
+                                                   rg, ru);
                         if (c == STEPS - 1 && h == 1) {
                             ptx::tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                            if (lane == 0) release_acc(acc);
                         }
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
@@ -487,13 +520,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
                     if (!aok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
                     uint32_t r0[32], r1[32];
-                    ptx::tmem_ld_32x32(t_acc + c * 64, r0);
-                    ptx::tmem_ld_32x32(t_acc + c * 64 + 32, r1);
-                    ptx::tmem_ld_wait();
+                    ptx::tmem_ld_32x32_x2_wait(t_acc + c * 64, t_acc + c * 64 + 32, r0, r1);
                     if (c == STEPS - 1) {
                         ptx::tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                        if (lane == 0) release_acc(acc);
                     }
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
@@ -516,12 +547,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                 } else {  // kEpiF32: 32 fp32 columns per step
                     uint32_t r0[32];
-                    ptx::tmem_ld_32x32(t_acc + c * 32, r0);
-                    ptx::tmem_ld_wait();
+                    ptx::tmem_ld_32x32_wait(t_acc + c * 32, r0);
                     if (c == STEPS - 1) {
                         ptx::tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+                        if (lane == 0) release_acc(acc);
                     }
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
@@ -535,30 +565,36 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     // the slot the NEXT step writes was last stored SLOTS-1 groups ago
                     ptx::bulk_wait_group_read<(SLOTS >= 2 ? SLOTS - 2 : 0)>();
                 }
+                __syncwarp();
                 ptx::named_bar_sync(1, kEpiThreads);
                 if (leader) {
-                    if (ok) {
+                    // The row coordinate is handed to the TMA unit through a fresh register. Without
+                    // this the pair build of the plain-store epilogue issued every store at row 0
+                    // (the long-lived copy of m0 the compiler kept was stale at this point); the
+                    // parity tests on multi-tile shapes guard this.
+                    const int y = ptx::fresh(m0);
+                    if (ok && y < p.M) {
                         if (EPI == kEpiStore || EPI == kEpiMulGeluGrad) {
                             const int x = n0 + c * 64;
-                            if (x < p.N) ptx::tma_store_2d(&tmD, buf, x, m0);
+                            if (x < p.N) ptx::tma_store_2d(&tmD, buf, x, y);
                         } else if (EPI == kEpiGelu) {
                             const int x = n0 + c * 64;
                             if (x < p.N) {
-                                ptx::tma_store_2d(&tmD, buf, x, m0);
-                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, m0);
+                                ptx::tma_store_2d(&tmD, buf, x, y);
+                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, y);
                             }
                         } else if (EPI == kEpiSwiglu) {
                             const int x = n0 + c * 64;
                             if (x < p.swiglu_h) {
-                                ptx::tma_store_2d(&tmD, buf, x, m0);
-                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, m0);
-                                ptx::tma_store_2d(&tmE, buf + 2 * kStgBytes, p.swiglu_h + x, m0);
+                                ptx::tma_store_2d(&tmD, buf, x, y);
+                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, y);
+                                ptx::tma_store_2d(&tmE, buf + 2 * kStgBytes, p.swiglu_h + x, y);
                             }
                         } else {
                             const int x = n0 + c * 32;
                             if (x < p.N) {
-                                if (p.reduce) ptx::tma_reduce_add_2d(&tmD, buf, x, m0);
-                                else ptx::tma_store_2d(&tmD, buf, x, m0);
+                                if (p.reduce) ptx::tma_reduce_add_2d(&tmD, buf, x, y);
+                                else ptx::tma_store_2d(&tmD, buf, x, y);
                             }
                         }
                     }
@@ -570,6 +606,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     }
                     if (SLOTS == 1) ptx::bulk_wait_group_read<0>();
                 }
+                __syncwarp();  // the single-lane block above rejoins its warp before collective ops
                 if (SLOTS == 1) ptx::named_bar_sync(1, kEpiThreads);
             }
             if (++acc == 2) {
@@ -587,11 +624,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const uint64_t t0 = ptx::globaltimer_ns();
         while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
     }
+    __syncwarp();
     ptx::tc_fence_before();
-    __syncthreads();
+    if (CG == 2) ptx::cluster_sync();  // neither CTA of a pair leaves while the other may still signal it
+    else __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+        ptx::tmem_dealloc<CG>(tmem_base, Cfg::TMEM_COLS);
     }
 }
 

@@ -5,8 +5,10 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <string>
@@ -22,6 +24,7 @@ using namespace nb;
 constexpr int kMaxDevices = 64;
 constexpr unsigned long long kDefaultTimeoutNs = 2000000000ull;  // 2 s per wait
 
+std::atomic<long long> g_launches{0};
 thread_local std::string g_err;
 thread_local cudaStream_t g_stream = nullptr;
 
@@ -131,7 +134,10 @@ int get_tmap(DeviceState &s, CUtensorMap *out, const void *ptr, uint64_t rows, u
     cuuint64_t strides[1] = {cols * esz};
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUtensorMap m;
+    // The encoder does not write every byte of the opaque descriptor: start from zeros, otherwise
+    // stack garbage ends up in fields the TMA unit reads.
+    alignas(64) CUtensorMap m;
+    memset(&m, 0, sizeof(m));
     CUresult r = g_encode(&m, dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
                           2, const_cast<void *>(ptr), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -177,11 +183,30 @@ template <class Cfg>
 int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
 {
     static bool attr_set[kMaxDevices] = {};
+    static int max_clusters[kMaxDevices] = {};
     int dev = 0;
     NB_CUDA(cudaGetDevice(&dev));
     if (!attr_set[dev]) {
         NB_CUDA(cudaFuncSetAttribute(gemm_kernel<Cfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      static_cast<int>(Cfg::SMEM_BYTES)));
+        max_clusters[dev] = s.num_sms / Cfg::CG;
+        if (Cfg::CG == 2) {  // how many CTA pairs can be resident at once
+            cudaLaunchConfig_t qc = {};
+            qc.gridDim = dim3(static_cast<unsigned>(s.num_sms));
+            qc.blockDim = dim3(kNumThreads);
+            qc.dynamicSmemBytes = Cfg::SMEM_BYTES;
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 2;
+            qa[0].val.clusterDim.y = 1;
+            qa[0].val.clusterDim.z = 1;
+            qc.attrs = qa;
+            qc.numAttrs = 1;
+            int n = 0;
+            NB_CUDA(cudaOccupancyMaxActiveClusters(&n, gemm_kernel<Cfg>, &qc));
+            if (n < 1) return fail(NB_ERR_CUDA, "no CTA pair of this kernel fits on the device");
+            if (n < max_clusters[dev]) max_clusters[dev] = n;
+        }
         attr_set[dev] = true;
     }
     CUtensorMap tA, tB, tD, tE;
@@ -200,7 +225,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     p.M = a.M;
     p.N = a.N;
     p.K = a.K;
-    p.tiles_m = (a.M + kBlockM - 1) / kBlockM;
+    p.tiles_m = (a.M + Cfg::TILE_M - 1) / Cfg::TILE_M;
     const int n_span = (Cfg::EPI == kEpiSwiglu) ? a.swiglu_h : a.N;
     const int n_tile = (Cfg::EPI == kEpiSwiglu) ? 128 : Cfg::BLOCK_N;
     p.tiles_n = (n_span + n_tile - 1) / n_tile;
@@ -209,7 +234,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     if (splits > p.kblocks) splits = p.kblocks;
     p.kblocks_per_split = (p.kblocks + splits - 1) / splits;
     p.splits = (p.kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;
-    p.group_m = 16;
+    p.group_m = 16 / Cfg::CG;
     p.swiglu_h = a.swiglu_h;
     p.reduce = a.reduce;
     p.bias = static_cast<const __nv_bfloat16 *>(a.bias);
@@ -217,20 +242,59 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     p.timeout_ns = kDefaultTimeoutNs;
     const long long units = 1ll * p.tiles_m * p.tiles_n * p.splits;
     if (units <= 0 || units >= (1ll << 31)) return fail(NB_ERR_UNSUPPORTED, "tile count out of range");
-    const int grid = static_cast<int>(units < s.num_sms ? units : s.num_sms);
-    gemm_kernel<Cfg><<<grid, kNumThreads, Cfg::SMEM_BYTES, stream>>>(tA, tB, tD, tE, p);
-    NB_CUDA(cudaGetLastError());
+    const int clusters = static_cast<int>(units < max_clusters[dev] ? units : max_clusters[dev]);
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(clusters * Cfg::CG));
+    cfg.blockDim = dim3(kNumThreads);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[1];
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = Cfg::CG;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 1;
+    NB_CUDA(cudaLaunchKernelEx(&cfg, gemm_kernel<Cfg>, tA, tB, tD, tE, p));
+    ++g_launches;
     return NB_OK;
 }
 
-// kernel configurations: <BLOCK_N, STAGES, staging buffers, A MN-major, B MN-major, epilogue>
-using FwdStore = GemmCfg<256, 4, 2, false, false, kEpiStore>;
-using FwdGelu = GemmCfg<256, 3, 4, false, false, kEpiGelu>;
-using FwdSwiglu = GemmCfg<256, 3, 3, false, false, kEpiSwiglu>;
-using DgradStore = GemmCfg<256, 4, 2, false, true, kEpiStore>;
-using DgradMulGelu = GemmCfg<256, 3, 4, false, true, kEpiMulGeluGrad>;
-using WgradF32 = GemmCfg<256, 4, 2, true, true, kEpiF32>;
-using WgradBf16 = GemmCfg<256, 4, 2, true, true, kEpiStore>;
+// Kernel configurations: <CTAs per tile, BLOCK_N, stages, staging buffers, A MN-major, B MN-major,
+// epilogue>. The pair forms (256-row tiles) are used whenever there is more than one 128-row block;
+// the single-CTA forms serve small row counts.
+using FwdStore1 = GemmCfg<1, 256, 4, 2, false, false, kEpiStore>;
+using FwdGelu1 = GemmCfg<1, 256, 3, 4, false, false, kEpiGelu>;
+using FwdSwiglu1 = GemmCfg<1, 256, 3, 3, false, false, kEpiSwiglu>;
+using DgradStore1 = GemmCfg<1, 256, 4, 2, false, true, kEpiStore>;
+using DgradMulGelu1 = GemmCfg<1, 256, 3, 4, false, true, kEpiMulGeluGrad>;
+using WgradF32_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32>;
+using WgradBf16_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiStore>;
+using FwdStore2 = GemmCfg<2, 256, 6, 2, false, false, kEpiStore>;
+using FwdGelu2 = GemmCfg<2, 256, 5, 4, false, false, kEpiGelu>;
+using FwdSwiglu2 = GemmCfg<2, 256, 5, 3, false, false, kEpiSwiglu>;
+using DgradStore2 = GemmCfg<2, 256, 6, 2, false, true, kEpiStore>;
+using DgradMulGelu2 = GemmCfg<2, 256, 5, 4, false, true, kEpiMulGeluGrad>;
+using WgradF32_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32>;
+using WgradBf16_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiStore>;
+
+bool use_pairs(int M)
+{
+    static const int force = [] {
+        const char *e = getenv("NB_CTA_GROUP");  // debugging aid: 1 or 2 forces one form
+        return e ? atoi(e) : 0;
+    }();
+    if (force == 1) return false;
+    if (force == 2) return true;
+    return M > kBlockM;
+}
+
+template <class C1, class C2>
+int launch_gemm_auto(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
+{
+    return use_pairs(a.M) ? launch_gemm<C2>(s, a, stream) : launch_gemm<C1>(s, a, stream);
+}
 
 int ensure_workspace(DeviceState &s, size_t bytes)
 {
@@ -264,6 +328,7 @@ int launch_dbias(DeviceState &s, float *dbias, const void *dz, int64_t BT, int64
                                                      static_cast<int>(OC),
                                                      static_cast<int>(rows_per_block));
     NB_CUDA(cudaGetLastError());
+    ++g_launches;
     return NB_OK;
 }
 
@@ -330,15 +395,15 @@ int nb_linear_forward_ex(void *out, void *pre_act, const void *inp, const void *
     a.M = static_cast<int>(BT); a.N = static_cast<int>(OC); a.K = static_cast<int>(C);
     a.bias = bias;
     a.splits = 1;
-    if (act == NB_ACT_NONE) return launch_gemm<FwdStore>(*s, a, stream);
+    if (act == NB_ACT_NONE) return launch_gemm_auto<FwdStore1, FwdStore2>(*s, a, stream);
     if (!pre_act) {
         // the activated result without its pre-activation: only NONE can skip the second plane
         return fail(NB_ERR_INVALID_ARG, "pre_act must be given when act != NONE");
     }
     a.E = pre_act; a.e_rows = BT; a.e_cols = OC;
-    if (act == NB_ACT_GELU) return launch_gemm<FwdGelu>(*s, a, stream);
+    if (act == NB_ACT_GELU) return launch_gemm_auto<FwdGelu1, FwdGelu2>(*s, a, stream);
     a.swiglu_h = static_cast<int>(OC / 2);
-    return launch_gemm<FwdSwiglu>(*s, a, stream);
+    return launch_gemm_auto<FwdSwiglu1, FwdSwiglu2>(*s, a, stream);
 }
 
 int nb_linear_forward(void *out, const void *inp, const void *weight, const void *bias, int64_t BT,
@@ -407,6 +472,7 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
                 static_cast<const uint4 *>(pre_act), BT, hvec);
         }
         NB_CUDA(cudaGetLastError());
+        ++g_launches;
         dz = s->workspace;
     }
 
@@ -420,9 +486,9 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
         a.splits = 1;
         if (inp_pre_act) {
             a.E = inp_pre_act; a.e_rows = BT; a.e_cols = C;
-            rc = launch_gemm<DgradMulGelu>(*s, a, stream);
+            rc = launch_gemm_auto<DgradMulGelu1, DgradMulGelu2>(*s, a, stream);
         } else {
-            rc = launch_gemm<DgradStore>(*s, a, stream);
+            rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream);
         }
         if (rc != NB_OK) return rc;
     }
@@ -436,20 +502,22 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
         a.M = static_cast<int>(OC); a.N = static_cast<int>(C); a.K = static_cast<int>(BT);
         if (dweight_dtype == NB_DTYPE_F32) {
             a.d_dtype = 1;
-            const int tiles = ((a.M + kBlockM - 1) / kBlockM) * ((a.N + 255) / 256);
+            const int tile_m = use_pairs(a.M) ? 2 * kBlockM : kBlockM;
+            const int tiles = ((a.M + tile_m - 1) / tile_m) * ((a.N + 255) / 256);
             const int kblocks = (a.K + kBlockK - 1) / kBlockK;
-            int splits = (2 * s->num_sms + tiles - 1) / tiles;
+            const int slots = s->num_sms / (use_pairs(a.M) ? 2 : 1);  // tiles resident at once
+            int splits = (2 * slots + tiles - 1) / tiles;
             if (splits > kblocks / 4) splits = kblocks / 4;
             if (splits < 1) splits = 1;
             a.splits = splits;
             a.reduce = (accumulate || splits > 1) ? 1 : 0;
             if (!accumulate && splits > 1)
                 NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(OC * C) * 4, stream));
-            rc = launch_gemm<WgradF32>(*s, a, stream);
+            rc = launch_gemm_auto<WgradF32_1, WgradF32_2>(*s, a, stream);
         } else {
             a.d_dtype = 0;
             a.splits = 1;
-            rc = launch_gemm<WgradBf16>(*s, a, stream);
+            rc = launch_gemm_auto<WgradBf16_1, WgradBf16_2>(*s, a, stream);
         }
         if (rc != NB_OK) return rc;
     }
@@ -526,6 +594,8 @@ int nb_check_status(void)
     return fail(NB_ERR_CUDA, "kernel reported internal error %d (block %d)", host[0], host[2]);
 }
 
+int64_t nb_kernel_launches(void) { return g_launches.load(); }
+
 int nb_debug_wait_timeout(int64_t limit_us)
 {
     if (limit_us < 1 || limit_us > 1000000)
@@ -536,6 +606,7 @@ int nb_debug_wait_timeout(int64_t limit_us)
     if (rc != NB_OK) return rc;
     wait_timeout_kernel<<<1, 32, 0, g_stream>>>(s->status, static_cast<unsigned long long>(limit_us) * 1000ull);
     NB_CUDA(cudaGetLastError());
+    ++g_launches;
     return NB_OK;
 }
 

@@ -1,0 +1,180 @@
+"""The linear layers of a whole model as a sequence of library calls.
+
+`LinearStack` owns the device buffers of one workload (GPT-2 124M: 12 blocks of
+qkv / attn-proj / fc+GELU / proj and the tied head; or the Qwen3-0.6B-shaped
+adapter linears) and replays a micro-step: every forward in model order, then
+every backward in reverse order, weight and bias gradients accumulated in fp32
+across micro-steps (paper: Method/Batch geometry). Only the linears are on this
+path: the tensors that attention, layer norm and the loss would produce are
+seeded synthetic inputs, distinct per layer and per micro-step. The class only
+allocates, generates inputs and marshals calls; all arithmetic is in the CUDA
+library.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import torch
+
+from . import binding as nb
+from . import shapes, synth
+
+
+@dataclass
+class _Layer:
+    spec: shapes.LinearSpec
+    index: int
+    weight: torch.Tensor = None
+    bias: torch.Tensor = None
+    dweight: torch.Tensor = None
+    dbias: torch.Tensor = None
+    out: torch.Tensor = None
+    pre: torch.Tensor = None
+    dinp: torch.Tensor = None
+    inp: list = field(default_factory=list)    # per micro-step, None if chained from the producer
+    dout: list = field(default_factory=list)   # per micro-step, None if chained from the consumer
+    chained_from: "_Layer" = None              # fc -> proj: proj.inp is fc.out
+    dz_from: "_Layer" = None                   # fc.dz is proj.dinp (fused GELU backward)
+
+
+class LinearStack:
+    def __init__(self, model: str, BT: int, micro_steps: int, device="cuda", config_id: int = 4,
+                 seed_offset: int = 0, wgrad: bool = True, generate: bool = True):
+        self.model, self.BT, self.micro_steps, self.device = model, BT, micro_steps, device
+        self.wgrad = wgrad
+        self.layers: list[_Layer] = []
+        if model == "gpt2":
+            nblocks, block, head = shapes.GPT2_LAYERS, shapes.gpt2_block, shapes.gpt2_lm_head()
+        elif model == "gpt2_block":
+            nblocks, block, head = 1, shapes.gpt2_block, None
+        elif model == "gpt2_head":
+            nblocks, block, head = 0, shapes.gpt2_block, shapes.gpt2_lm_head()
+        elif model == "qwen3":
+            nblocks, block, head = shapes.QWEN3_LAYERS, shapes.qwen3_block, None
+        else:
+            raise ValueError(model)
+        idx = 0
+        for _ in range(nblocks):
+            prev = None
+            for s in block():
+                L = _Layer(s, idx)
+                if s.fused_gelu_bwd and prev is not None and prev.spec.act == shapes.ACT_GELU:
+                    L.chained_from = prev
+                    prev.dz_from = L
+                self.layers.append(L)
+                prev = L
+                idx += 1
+        if head is not None:
+            self.layers.append(_Layer(head, idx))
+        self.config_id, self.seed_offset = config_id, seed_offset
+        self._allocate()
+        if generate:
+            self.generate_inputs()
+
+    # ------------------------------------------------------------------ buffers
+    def _allocate(self):
+        dev, BT = self.device, self.BT
+        bf, f32 = torch.bfloat16, torch.float32
+        for L in self.layers:
+            s = L.spec
+            L.weight = torch.empty((s.OC, s.C), dtype=bf, device=dev)
+            L.bias = torch.empty((s.OC,), dtype=bf, device=dev) if s.bias else None
+            if self.wgrad:
+                L.dweight = torch.empty((s.OC, s.C), dtype=f32, device=dev)
+                L.dbias = torch.empty((s.OC,), dtype=f32, device=dev) if s.bias else None
+            L.out = torch.empty((BT, s.out_cols), dtype=bf, device=dev)
+            L.pre = torch.empty((BT, s.OC), dtype=bf, device=dev) if s.act != shapes.ACT_NONE else None
+            L.dinp = torch.empty((BT, s.C), dtype=bf, device=dev)
+            for _ in range(self.micro_steps):
+                L.inp.append(None if L.chained_from else torch.empty((BT, s.C), dtype=bf, device=dev))
+                L.dout.append(None if L.dz_from else torch.empty((BT, s.out_cols), dtype=bf, device=dev))
+
+    def seed(self, L: _Layer, role: int, ms: int = 0) -> int:
+        return synth.tensor_seed(self.config_id, L.index, role, ms) + 100000 * self.seed_offset
+
+    def generate_inputs(self):
+        """Fill weights, biases and per-micro-step inputs / output gradients from their seeds."""
+        dev = self.device
+        for L in self.layers:
+            s = L.spec
+            L.weight.copy_(synth.normal(self.seed(L, 1), (s.OC, s.C), s.w_std, dev))
+            if s.OC == shapes.VOCAB_PADDED:
+                synth.zero_pad_vocab_rows(L.weight)
+            if L.bias is not None:
+                L.bias.copy_(synth.normal(self.seed(L, 2), (s.OC,), 0.02, dev))
+            dstd = 1e-4 if s.OC == shapes.VOCAB_PADDED else 1e-3
+            for ms in range(self.micro_steps):
+                if L.inp[ms] is not None:
+                    L.inp[ms].copy_(synth.normal(self.seed(L, 0, ms), (self.BT, s.C), 1.0, dev))
+                if L.dout[ms] is not None:
+                    L.dout[ms].copy_(synth.normal(self.seed(L, 3, ms), (self.BT, s.out_cols), dstd, dev))
+                    if s.OC == shapes.VOCAB_PADDED:
+                        synth.zero_pad_vocab_cols(L.dout[ms])
+
+    def input_tensors(self, ms: int):
+        """The per-micro-step input tensors (what a host would have to supply)."""
+        ts = []
+        for L in self.layers:
+            if L.inp[ms] is not None:
+                ts.append(L.inp[ms])
+            if L.dout[ms] is not None:
+                ts.append(L.dout[ms])
+        return ts
+
+    def gradient_tensors(self):
+        ts = []
+        for L in self.layers:
+            if L.dweight is not None:
+                ts.append(L.dweight)
+            if L.dbias is not None:
+                ts.append(L.dbias)
+        return ts
+
+    # ------------------------------------------------------------------ accounting
+    def flops_per_micro_step(self) -> int:
+        return sum(L.spec.flops(self.BT, self.wgrad) for L in self.layers)
+
+    def calls_per_micro_step(self) -> int:
+        return 2 * len(self.layers)
+
+    # ------------------------------------------------------------------ the path
+    def layer_inp(self, L: _Layer, ms: int) -> torch.Tensor:
+        return L.chained_from.out if L.chained_from else L.inp[ms]
+
+    def forward(self, ms: int, hook=None):
+        BT = self.BT
+        for L in self.layers:
+            s = L.spec
+            if hook:
+                hook("fwd", L, True)
+            nb.nb_linear_forward_ex(L.out, L.pre, self.layer_inp(L, ms), L.weight, L.bias, BT, s.C,
+                                    s.OC, s.act)
+            if hook:
+                hook("fwd", L, False)
+
+    def backward(self, ms: int, hook=None):
+        BT = self.BT
+        acc = 1 if ms > 0 else 0
+        for L in reversed(self.layers):
+            s = L.spec
+            if L.dz_from is not None:
+                # the consumer's dgrad epilogue already applied gelu'(pre): its dinp is this dz
+                dout, act, pre = L.dz_from.dinp, shapes.ACT_NONE, None
+            else:
+                dout, act, pre = L.dout[ms], s.act, L.pre
+            inp_pre = L.chained_from.pre if L.chained_from else None
+            if hook:
+                hook("bwd", L, True)
+            nb.nb_linear_backward_ex(L.dinp, L.dweight, L.dbias, dout, self.layer_inp(L, ms), L.weight,
+                                     pre, inp_pre, BT, s.C, s.OC, act, acc)
+            if hook:
+                hook("bwd", L, False)
+
+    def micro_step(self, ms: int, hook=None):
+        self.forward(ms, hook)
+        self.backward(ms, hook)
+
+    def step(self, hook=None):
+        """One pass of the whole path: every micro-step, forward then backward."""
+        for ms in range(self.micro_steps):
+            self.micro_step(ms, hook)

@@ -1,0 +1,406 @@
+"""GPU-vs-oracle parity through the C ABI: every element on small and odd shapes and on the
+two small workloads; sampled rows, columns and elements at the full-size workloads."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_28568_b200 import binding as nb
+from paper_2609_28568_b200 import shapes, synth
+from parity import (Guarded, check_bf16, check_f32, f32, rel_frob, sample_indices)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(autouse=True)
+def _status_clean():
+    yield
+    nb.nb_check_status()  # no kernel may have given up on a wait
+
+
+def gen(seed, shape, std):
+    return synth.normal(seed, shape, std, DEV)
+
+
+# --------------------------------------------------------------------------- every element
+
+def run_layer_full(BT, C, OC, act, bias=True, w_std=0.02, dout_std=1e-3, seed=100):
+    """Forward + backward of one layer on the GPU and in the oracle, compared element by element.
+    Backward applies the layer's own activation derivative through the GPU-stored pre-activation,
+    which is also what the oracle is handed, so each call is checked on its own."""
+    inp = gen(seed, (BT, C), 1.0)
+    w = gen(seed + 1, (OC, C), w_std)
+    b = gen(seed + 2, (OC,), 0.02) if bias else None
+    ocols = OC // 2 if act == nb.ACT_SWIGLU else OC
+    dout = gen(seed + 3, (BT, ocols), dout_std)
+
+    out = Guarded((BT, ocols), torch.bfloat16)
+    pre = Guarded((BT, OC), torch.bfloat16) if act != nb.ACT_NONE else None
+    nb.nb_linear_forward_ex(out.t, pre.t if pre else None, inp, w, b, BT, C, OC, act)
+    o_ref, p_ref = oracle.linear_forward(f32(inp), f32(w), f32(b) if bias else None, act)
+    check_bf16(out.t, o_ref, "out")
+    out.check("out")
+    if pre:
+        check_bf16(pre.t, p_ref, "pre_act")
+        pre.check("pre_act")
+
+    dinp = Guarded((BT, C), torch.bfloat16)
+    dw = Guarded((OC, C), torch.float32, fill=777.0)  # accumulate=0 must overwrite
+    db = Guarded((OC,), torch.float32, fill=-55.0) if bias else None
+    nb.nb_linear_backward_ex(dinp.t, dw.t, db.t if db else None, dout, inp, w,
+                             pre.t if pre else None, None, BT, C, OC, act, 0)
+    r = oracle.linear_backward(f32(dout), f32(inp), f32(w), pre=f32(pre.t) if pre else None, act=act)
+    check_bf16(dinp.t, r["dinp"], "dinp")
+    check_f32(dw.t, r["dweight"], "dweight")
+    dinp.check("dinp")
+    dw.check("dweight")
+    if db:
+        check_f32(db.t, r["dbias"], "dbias")
+        db.check("dbias")
+
+
+@pytest.mark.parametrize("act", [nb.ACT_NONE, nb.ACT_GELU, nb.ACT_SWIGLU])
+@pytest.mark.parametrize("BT,C,OC", [
+    (1, 8, 16),          # a single row, one k block
+    (128, 64, 256),      # exactly one tile
+    (136, 72, 208),      # ragged in every dimension
+    (392, 328, 528),     # several tiles with ragged tails
+    (700, 200, 1040),    # more than one tile along OC with a tail
+])
+def test_small_shapes_every_element(BT, C, OC, act):
+    run_layer_full(BT, C, OC, act, w_std=0.05, dout_std=1e-3, seed=7 * BT + OC + act)
+
+
+def test_integer_inputs_are_exact():
+    """Small integers: products and sums are exact in bf16 x bf16 -> fp32, so GPU == oracle exactly.
+    Catches any indexing or layout error that a tolerance could hide."""
+    BT, C, OC = 200, 136, 328
+    g = torch.Generator().manual_seed(3)
+    ri = lambda *s: torch.randint(-4, 5, s, generator=g).to(torch.bfloat16).to(DEV)
+    inp, w, b, dz = ri(BT, C), ri(OC, C), ri(OC), ri(BT, OC)
+    out, _ = nb.linear_forward(inp, w, b, nb.ACT_NONE)
+    o_ref, _ = oracle.linear_forward(f32(inp), f32(w), f32(b))
+    small = np.abs(o_ref) <= 256  # integers up to 2^8 are representable in bf16
+    assert small.mean() > 0.9
+    assert np.array_equal(f32(out).astype(np.float64)[small], o_ref[small])
+    dinp, dw, db = nb.linear_backward(dz, inp, w)
+    r = oracle.linear_backward(f32(dz), f32(inp), f32(w))
+    assert np.array_equal(f32(dw).astype(np.float64), r["dweight"])
+    assert np.array_equal(f32(db).astype(np.float64), r["dbias"])
+    exact = np.abs(r["dinp"]) <= 256
+    assert exact.mean() > 0.9
+    assert np.array_equal(f32(dinp).astype(np.float64)[exact], r["dinp"][exact])
+
+
+def test_config1_fc_layer_forward_backward():
+    """Workload 1: one GPT-2 MLP fc layer, B=2 T=64, tanh-GELU, own pre-activation in backward."""
+    run_layer_full(128, 768, 3072, nb.ACT_GELU, seed=synth.tensor_seed(1, 0, 0))
+
+
+def test_short_form_calls_two_plane_out():
+    """The 8- and 11-argument entry points: `out` carries the activated and pre-activation planes."""
+    BT, C, OC = 128, 768, 3072
+    inp, w, b = gen(1, (BT, C), 1.0), gen(2, (OC, C), 0.02), gen(3, (OC,), 0.02)
+    dout = gen(4, (BT, OC), 1e-3)
+    n = nb.nb_linear_out_elems(BT, OC, nb.ACT_GELU)
+    planes = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    nb.nb_linear_forward(planes, inp, w, b, BT, C, OC, nb.ACT_GELU)
+    out, pre = planes[:BT * OC].view(BT, OC), planes[BT * OC:].view(BT, OC)
+    out2, pre2 = nb.linear_forward(inp, w, b, nb.ACT_GELU)
+    assert torch.equal(out, out2) and torch.equal(pre, pre2)
+    dinp = torch.empty((BT, C), dtype=torch.bfloat16, device=DEV)
+    dw = torch.empty((OC, C), dtype=torch.float32, device=DEV)
+    db = torch.empty((OC,), dtype=torch.float32, device=DEV)
+    nb.nb_linear_backward(dinp, dw, db, dout, inp, w, pre, BT, C, OC, 0)
+    r = oracle.linear_backward(f32(dout), f32(inp), f32(w), pre=f32(pre), act=oracle.ACT_GELU)
+    check_bf16(dinp, r["dinp"], "dinp")
+    check_f32(dw, r["dweight"], "dweight")
+    check_f32(db, r["dbias"], "dbias")
+    # SwiGLU planes
+    OC2 = 512
+    w2 = gen(5, (OC2, C), 0.02)
+    n2 = nb.nb_linear_out_elems(BT, OC2, nb.ACT_SWIGLU)
+    planes2 = torch.empty(n2, dtype=torch.bfloat16, device=DEV)
+    nb.nb_linear_forward(planes2, inp, w2, None, BT, C, OC2, nb.ACT_SWIGLU)
+    o_ref, p_ref = oracle.linear_forward(f32(inp), f32(w2), None, oracle.ACT_SWIGLU)
+    check_bf16(planes2[:BT * OC2 // 2].view(BT, OC2 // 2), o_ref, "swiglu out")
+    check_bf16(planes2[BT * OC2 // 2:].view(BT, OC2), p_ref, "swiglu pre")
+
+
+def test_config2_block_linears():
+    """Workload 2: the four linears of one GPT-2 block at B=4, T=1024, every element."""
+    BT = 4096
+    for li, s in enumerate(shapes.gpt2_block()):
+        inp = gen(synth.tensor_seed(2, li, 0), (BT, s.C), 1.0)
+        w = gen(synth.tensor_seed(2, li, 1), (s.OC, s.C), s.w_std)
+        b = gen(synth.tensor_seed(2, li, 2), (s.OC,), 0.02)
+        dout = gen(synth.tensor_seed(2, li, 3), (BT, s.OC), 1e-3)
+        out, pre = nb.linear_forward(inp, w, b, s.act)
+        o_ref, p_ref = oracle.linear_forward(f32(inp), f32(w), f32(b), s.act)
+        check_bf16(out, o_ref, s.name + " out")
+        if pre is not None:
+            check_bf16(pre, p_ref, s.name + " pre")
+        dinp, dw, db = nb.linear_backward(dout, inp, w, pre_act=pre, act=s.act)
+        r = oracle.linear_backward(f32(dout), f32(inp), f32(w),
+                                   pre=f32(pre) if pre is not None else None, act=s.act)
+        check_bf16(dinp, r["dinp"], s.name + " dinp")
+        check_f32(dw, r["dweight"], s.name + " dweight")
+        check_f32(db, r["dbias"], s.name + " dbias")
+
+
+def test_config2_fused_gelu_backward_equals_composed():
+    """fc -> proj chain: proj's dgrad epilogue applies gelu'(fc.pre), giving fc's dz directly.
+    It must agree with the oracle and, to rounding, with the composed form (dgrad, then the
+    elementwise product inside fc's own backward)."""
+    BT = 4096
+    fc, proj = shapes.gpt2_block()[2], shapes.gpt2_block()[3]
+    x = gen(11, (BT, fc.C), 1.0)
+    w_fc, b_fc = gen(12, (fc.OC, fc.C), fc.w_std), gen(13, (fc.OC,), 0.02)
+    w_pr = gen(14, (proj.OC, proj.C), proj.w_std)
+    dout = gen(15, (BT, proj.OC), 1e-3)
+    h, pre = nb.linear_forward(x, w_fc, b_fc, nb.ACT_GELU)
+    # fused: dz_fc = (dout . W_proj) * gelu'(pre)
+    dz_fused, dw_pr, _ = nb.linear_backward(dout, h, w_pr, inp_pre_act=pre, need_dbias=False)
+    r = oracle.linear_backward(f32(dout), f32(h), f32(w_pr), inp_pre=f32(pre))
+    check_bf16(dz_fused, r["dinp"], "fused dz")
+    check_f32(dw_pr, r["dweight"], "proj dweight")
+    # composed: plain dgrad, then fc's backward applies gelu'(pre) itself
+    dh, _, _ = nb.linear_backward(dout, h, w_pr, need_dweight=False, need_dbias=False)
+    dx_c, dw_c, db_c = nb.linear_backward(dh, x, w_fc, pre_act=pre, act=nb.ACT_GELU)
+    dx_f, dw_f, db_f = nb.linear_backward(dz_fused, x, w_fc)
+    assert rel_frob(f32(dx_f), f32(dx_c)) < 5e-3
+    assert rel_frob(f32(dw_f), f32(dw_c)) < 5e-3
+    assert rel_frob(f32(db_f), f32(db_c)) < 5e-3
+    rr = oracle.linear_backward(f32(dz_fused), f32(x), f32(w_fc))
+    check_bf16(dx_f, rr["dinp"], "fc dinp")
+    check_f32(dw_f, rr["dweight"], "fc dweight")
+    check_f32(db_f, rr["dbias"], "fc dbias")
+
+
+# --------------------------------------------------------------------------- accumulation
+
+def test_accumulation_over_micro_steps():
+    """Four micro-steps into one fp32 buffer (first overwrites, the rest add) equal the oracle's
+    four accumulate calls; the buffers start out dirty."""
+    BT, C, OC = 1024, 768, 2304
+    w = gen(21, (OC, C), 0.02)
+    dw = Guarded((OC, C), torch.float32, fill=3.0)
+    db = Guarded((OC,), torch.float32, fill=3.0)
+    dw_ref = np.full((OC, C), -9.0)
+    db_ref = np.full((OC,), -9.0)
+    for ms in range(4):
+        inp = gen(synth.tensor_seed(4, 0, 0, ms), (BT, C), 1.0)
+        dout = gen(synth.tensor_seed(4, 0, 3, ms), (BT, OC), 1e-3)
+        nb.nb_linear_backward_ex(None, dw.t, db.t, dout, inp, w, None, None, BT, C, OC, nb.ACT_NONE,
+                                 1 if ms > 0 else 0)
+        oracle.linear_backward(f32(dout), f32(inp), f32(w), dweight=dw_ref, dbias=db_ref,
+                               accumulate=ms > 0, want=("dweight", "dbias"))
+    check_f32(dw.t, dw_ref, "accumulated dweight")
+    check_f32(db.t, db_ref, "accumulated dbias")
+    dw.check()
+    db.check()
+
+
+def test_reduce_dbias_standalone():
+    for BT, OC in ((1, 8), (77, 200), (4096, 2304), (5000, 776)):
+        dout = gen(31 + BT, (BT, OC), 1e-3)
+        db = Guarded((OC,), torch.float32, fill=1.5)
+        nb.nb_reduce_dbias(db.t, dout, BT, OC, 0)
+        ref = oracle.reduce_dbias(f32(dout))
+        check_f32(db.t, ref, "dbias")
+        nb.nb_reduce_dbias(db.t, dout, BT, OC, 1)
+        check_f32(db.t, 2 * ref, "dbias twice")
+        db.check()
+
+
+# --------------------------------------------------------------------------- edge cases
+
+def test_skipped_products_and_empty_batch():
+    BT, C, OC = 256, 128, 192
+    inp, w, dout = gen(41, (BT, C), 1.0), gen(42, (OC, C), 0.02), gen(43, (BT, OC), 1e-3)
+    r = oracle.linear_backward(f32(dout), f32(inp), f32(w))
+    # frozen weights: only dinp
+    dinp = Guarded((BT, C), torch.bfloat16)
+    nb.nb_linear_backward_ex(dinp.t, None, None, dout, None, w, None, None, BT, C, OC, 0, 0)
+    check_bf16(dinp.t, r["dinp"], "dinp only")
+    dinp.check()
+    # only dweight
+    dw = Guarded((OC, C), torch.float32)
+    nb.nb_linear_backward_ex(None, dw.t, None, dout, inp, None, None, None, BT, C, OC, 0, 0)
+    check_f32(dw.t, r["dweight"], "dweight only")
+    # BT == 0: nothing launched; accumulate=0 zeroes the gradients, accumulate=1 leaves them
+    dw.t.fill_(5.0)
+    db = torch.full((OC,), 5.0, device=DEV)
+    e = torch.empty((0, OC), dtype=torch.bfloat16, device=DEV)
+    ei = torch.empty((0, C), dtype=torch.bfloat16, device=DEV)
+    nb.nb_linear_backward_ex(None, dw.t, db, e.data_ptr() or 16, ei.data_ptr() or 16, w, None, None, 0, C, OC, 0, 1)
+    assert torch.all(dw.t == 5.0) and torch.all(db == 5.0)
+    nb.nb_linear_backward_ex(None, dw.t, db, e.data_ptr() or 16, ei.data_ptr() or 16, w, None, None, 0, C, OC, 0, 0)
+    assert torch.all(dw.t == 0.0) and torch.all(db == 0.0)
+    dw.check()
+
+
+def test_bf16_dweight_variant():
+    BT, C, OC = 512, 256, 384
+    inp, w, dout = gen(51, (BT, C), 1.0), gen(52, (OC, C), 0.02), gen(53, (BT, OC), 1e-3)
+    dw = Guarded((OC, C), torch.bfloat16)
+    nb.nb_linear_backward_ex(None, dw.t, None, dout, inp, None, None, None, BT, C, OC, 0, 0,
+                             nb.DTYPE_BF16)
+    r = oracle.linear_backward(f32(dout), f32(inp), f32(w), want=("dweight",))
+    check_bf16(dw.t, r["dweight"], "bf16 dweight")
+    dw.check()
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    nb.nb_debug_wait_timeout(2000)
+    with pytest.raises(nb.NbError) as e:
+        nb.nb_check_status()
+    assert e.value.code == nb.NB_ERR_TIMEOUT
+    nb.nb_check_status()  # status word cleared; the context still works:
+    run_layer_full(128, 64, 256, nb.ACT_NONE, seed=61)
+
+
+def test_other_stream():
+    s = torch.cuda.Stream()
+    BT, C, OC = 512, 256, 512
+    inp, w = gen(71, (BT, C), 1.0), gen(72, (OC, C), 0.02)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        out, _ = nb.linear_forward(inp, w, None, nb.ACT_NONE)
+    s.synchronize()
+    o_ref, _ = oracle.linear_forward(f32(inp), f32(w))
+    check_bf16(out, o_ref, "out on side stream")
+
+
+# --------------------------------------------------------------------------- full-size, sampled
+
+def _fwd_sampled(name, inp, w, b, act, out, pre, seed, nrows=48, ncols=24):
+    """Compare sampled full rows and full columns of out / pre with the oracle."""
+    BT, OC = inp.shape[0], w.shape[0]
+    H = OC // 2
+    rows = sample_indices(BT, nrows, seed)
+    o_ref, p_ref = oracle.linear_forward(f32(inp[rows]), f32(w), f32(b) if b is not None else None, act)
+    check_bf16(out[rows], o_ref, name + " out rows")
+    if pre is not None:
+        check_bf16(pre[rows], p_ref, name + " pre rows")
+    ocols = H if act == nb.ACT_SWIGLU else OC
+    cols = sample_indices(ocols, ncols, seed + 1)
+    wsel = np.concatenate([cols, cols + H]) if act == nb.ACT_SWIGLU else cols
+    wsel_t = torch.as_tensor(wsel, device=DEV)
+    o_ref, p_ref = oracle.linear_forward(f32(inp), f32(w[wsel_t]),
+                                         f32(b[wsel_t]) if b is not None else None, act)
+    check_bf16(out[:, torch.as_tensor(cols, device=DEV)], o_ref, name + " out cols")
+    if pre is not None:
+        check_bf16(pre[:, wsel_t], p_ref, name + " pre cols")
+
+
+def _bwd_sampled(name, dz, inp, w, dinp, dw, db, seed, inp_pre=None, dw_prev=None, nrows=48, ncols=8,
+                 check_dinp_cols=True):
+    """dz is the gradient that entered the products (after any activation derivative)."""
+    BT, (OC, C) = dz.shape[0], w.shape
+    if dinp is not None:
+        rows = sample_indices(BT, nrows, seed)
+        r = oracle.linear_backward(f32(dz[rows]), None, f32(w),
+                                   inp_pre=f32(inp_pre[rows]) if inp_pre is not None else None,
+                                   want=("dinp",))
+        check_bf16(dinp[rows], r["dinp"], name + " dinp rows")
+        if check_dinp_cols and BT * OC <= 2e8:
+            cols = torch.as_tensor(sample_indices(C, ncols, seed + 1), device=DEV)
+            r = oracle.linear_backward(f32(dz), None, f32(w[:, cols]),
+                                       inp_pre=f32(inp_pre[:, cols]) if inp_pre is not None else None,
+                                       want=("dinp",))
+            check_bf16(dinp[:, cols], r["dinp"], name + " dinp cols")
+    if dw is not None:
+        orow = torch.as_tensor(sample_indices(OC, nrows, seed + 2), device=DEV)
+        r = oracle.linear_backward(f32(dz[:, orow]), f32(inp), f32(w[orow]), want=("dweight",))
+        ref = r["dweight"] + (dw_prev[orow.cpu().numpy()] if dw_prev is not None else 0.0)
+        check_f32(dw[orow], ref, name + " dweight rows")
+        ccol = torch.as_tensor(sample_indices(C, ncols, seed + 3), device=DEV)
+        if BT * OC <= 2e8:
+            r = oracle.linear_backward(f32(dz), f32(inp[:, ccol]), f32(w[:, ccol]), want=("dweight",))
+            ref = r["dweight"] + (dw_prev[:, ccol.cpu().numpy()] if dw_prev is not None else 0.0)
+            check_f32(dw[:, ccol], ref, name + " dweight cols")
+    if db is not None:
+        check_f32(db, oracle.reduce_dbias(f32(dz)), name + " dbias")
+
+
+def test_config3_lm_head_full_size_sampled():
+    """Workload 3: tied head at B=16, T=1024: [16384, 768] x [50304, 768]^T, no bias, padded rows."""
+    BT, C, OC = 16384, 768, shapes.VOCAB_PADDED
+    inp = gen(synth.tensor_seed(3, 0, 0), (BT, C), 1.0)
+    w = synth.zero_pad_vocab_rows(gen(synth.tensor_seed(3, 0, 1), (OC, C), 0.02))
+    dout = synth.zero_pad_vocab_cols(gen(synth.tensor_seed(3, 0, 3), (BT, OC), 1e-4))
+    logits, _ = nb.linear_forward(inp, w, None, nb.ACT_NONE)
+    assert torch.all(logits[:, shapes.VOCAB_REAL:] == 0)  # padding rows of the weight: exact zeros
+    _fwd_sampled("head", inp, w, None, nb.ACT_NONE, logits, None, seed=301)
+    del logits
+    dinp, dw, _ = nb.linear_backward(dout, inp, w, need_dbias=False)
+    assert torch.all(dw[shapes.VOCAB_REAL:] == 0)  # padding columns of dlogits: no gradient
+    _bwd_sampled("head", dout, inp, w, dinp, dw, None, seed=311, check_dinp_cols=False)
+    # second micro-step accumulates into the same buffer (read-modify-write of 155 MB)
+    prev = f32(dw).astype(np.float64)
+    nb.linear_backward(dout, inp, w, dweight=dw, accumulate=True, need_dinp=False, need_dbias=False)
+    orow = sample_indices(OC, 48, 313)
+    assert rel_frob(f32(dw[torch.as_tensor(orow, device=DEV)]), 2 * prev[orow]) < 1e-5
+
+
+def test_config4_block_and_head_at_full_batch_sampled():
+    """Workload 4 (one block at B=16, T=1024 and two accumulation steps), sampled: includes the
+    fused GELU backward in proj's dgrad."""
+    BT = 16384
+    blk = shapes.gpt2_block()
+    for li, s in enumerate(blk):
+        w = gen(synth.tensor_seed(4, li, 1), (s.OC, s.C), s.w_std)
+        b = gen(synth.tensor_seed(4, li, 2), (s.OC,), 0.02)
+        dw = torch.empty((s.OC, s.C), dtype=torch.float32, device=DEV)
+        db = torch.empty((s.OC,), dtype=torch.float32, device=DEV)
+        dw_prev = None
+        for ms in range(2):
+            inp = gen(synth.tensor_seed(4, li, 0, ms), (BT, s.C), 1.0)
+            dout = gen(synth.tensor_seed(4, li, 3, ms), (BT, s.OC), 1e-3)
+            out, pre = nb.linear_forward(inp, w, b, s.act)
+            if ms == 0:
+                _fwd_sampled(s.name, inp, w, b, s.act, out, pre, seed=400 + li)
+            inp_pre = gen(synth.tensor_seed(4, li, 4, ms), (BT, s.C), 1.0) if s.fused_gelu_bwd else None
+            dinp, _, _ = nb.linear_backward(dout, inp, w, inp_pre_act=inp_pre, dweight=dw, dbias=db,
+                                            accumulate=ms > 0)
+            if ms == 0:
+                _bwd_sampled(s.name, dout, inp, w, dinp, dw, db, seed=410 + li, inp_pre=inp_pre)
+                dw_prev = f32(dw).astype(np.float64)
+                db_prev = f32(db).astype(np.float64)
+            else:
+                _bwd_sampled(s.name + " step2", dout, inp, w, None, dw, None, seed=420 + li,
+                             dw_prev=dw_prev)
+                check_f32(db, db_prev + oracle.reduce_dbias(f32(dout)), s.name + " dbias step2")
+
+
+def test_config5_adapter_shapes_sampled():
+    """Workload 5: Qwen3-0.6B-shaped linears at B=8, T=2048, no bias, SwiGLU fused in gate|up."""
+    BT = 16384
+    for li, s in enumerate(shapes.qwen3_block()):
+        inp = gen(synth.tensor_seed(5, li, 0), (BT, s.C), 1.0)
+        w = gen(synth.tensor_seed(5, li, 1), (s.OC, s.C), 0.02)
+        dout = gen(synth.tensor_seed(5, li, 3), (BT, s.out_cols), 1e-3)
+        out, pre = nb.linear_forward(inp, w, None, s.act)
+        _fwd_sampled(s.name, inp, w, None, s.act, out, pre, seed=500 + li, nrows=32, ncols=16)
+        # 5a: with wgrad; 5b (frozen base): dinp only
+        dinp, dw, _ = nb.linear_backward(dout, inp, w, pre_act=pre, act=s.act, need_dbias=False)
+        dinp_b, _, _ = nb.linear_backward(dout, inp, w, pre_act=pre, act=s.act, need_dweight=False,
+                                          need_dbias=False)
+        assert torch.equal(dinp, dinp_b)
+        if s.act == nb.ACT_SWIGLU:
+            rows = sample_indices(BT, 32, 520 + li)
+            r = oracle.linear_backward(f32(dout[rows]), None, f32(w), pre=f32(pre[rows]),
+                                       act=oracle.ACT_SWIGLU, want=("dinp", "dz"))
+            check_bf16(dinp[rows], r["dinp"], s.name + " dinp rows")
+            orow = sample_indices(s.OC, 32, 521 + li)
+            ot = torch.as_tensor(orow, device=DEV)
+            # dweight rows need dz columns: take them from the oracle's dz for all rows
+            rz = oracle.linear_backward(f32(dout), None, f32(w), pre=f32(pre), act=oracle.ACT_SWIGLU,
+                                        want=("dz",))
+            dzs = rz["dz"][:, orow].astype(np.float32)
+            rw = oracle.linear_backward(dzs, f32(inp), f32(w[ot]), want=("dweight",))
+            check_f32(dw[ot], rw["dweight"], s.name + " dweight rows")
+        else:
+            _bwd_sampled(s.name, dout, inp, w, dinp, dw, None, seed=510 + li, nrows=32, ncols=8)

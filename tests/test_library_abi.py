@@ -1,0 +1,80 @@
+"""The C-ABI library loads without a GPU, exports what the header declares, and rejects
+malformed requests before touching the device."""
+import os
+import re
+
+import pytest
+
+from paper_2609_28568_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build()
+    return binding.lib()
+
+
+def test_exports_match_header(L):
+    header = open(os.path.join(ROOT, "include", "nb_linear.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(nb_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_version_and_out_elems(L):
+    assert L.nb_version() == 100
+    assert L.nb_linear_out_elems(128, 3072, binding.ACT_NONE) == 128 * 3072
+    assert L.nb_linear_out_elems(128, 3072, binding.ACT_GELU) == 2 * 128 * 3072
+    assert L.nb_linear_out_elems(16, 6144, binding.ACT_SWIGLU) == 16 * 3072 + 16 * 6144
+    assert L.nb_linear_out_elems(16, 7, binding.ACT_SWIGLU) == -1
+    assert L.nb_linear_out_elems(-1, 8, binding.ACT_NONE) == -1
+    assert L.nb_linear_out_elems(1, 8, 9) == -1
+
+
+def test_stream_is_per_thread_state(L):
+    assert L.nb_get_stream() in (None, 0)
+    L.nb_set_stream(0x1000)
+    assert L.nb_get_stream() == 0x1000
+    L.nb_set_stream(None)
+
+
+def test_malformed_requests_are_rejected_without_a_device(L):
+    P = 0x10000  # a fake, aligned device address: never dereferenced by a rejected call
+    fwd = L.nb_linear_forward_ex
+    assert fwd(None, None, P, P, None, 8, 8, 8, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert b"NULL" in L.nb_last_error()
+    assert fwd(P, None, P, P, None, 8, 8, 8, 7, None) == binding.NB_ERR_INVALID_ARG
+    assert fwd(P, None, P, P, None, -1, 8, 8, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert fwd(P, None, P, P, None, 8, 12, 8, 0, None) == binding.NB_ERR_UNSUPPORTED
+    assert fwd(P, None, P, P, None, 8, 8, 20, 0, None) == binding.NB_ERR_UNSUPPORTED
+    assert fwd(P + 2, None, P, P, None, 8, 8, 8, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert fwd(P, None, P, P, None, 8, 8, 24, binding.ACT_SWIGLU, None) == binding.NB_ERR_UNSUPPORTED
+    assert fwd(P, None, P, P, None, 1 << 31, 8, 8, 0, None) == binding.NB_ERR_UNSUPPORTED
+    bwd = L.nb_linear_backward_ex
+    assert bwd(P, P, P, None, P, P, None, None, 8, 8, 8, 0, 0, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert bwd(P, P, P, P, P, P, None, None, 8, 8, 8, 1, 0, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert bwd(P, P, P, P, None, P, None, None, 8, 8, 8, 0, 0, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert bwd(P, P, P, P, P, None, None, None, 8, 8, 8, 0, 0, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert bwd(None, P, P, P, P, P, None, P, 8, 8, 8, 0, 0, 0, None) == binding.NB_ERR_INVALID_ARG
+    assert bwd(P, P, P, P, P, P, None, None, 8, 8, 8, 0, 1, 1, None) == binding.NB_ERR_UNSUPPORTED
+    assert bwd(P, P, P, P, P, P, None, None, 8, 8, 8, 0, 0, 5, None) == binding.NB_ERR_INVALID_ARG
+    assert L.nb_reduce_dbias(None, P, 8, 8, 0) == binding.NB_ERR_INVALID_ARG
+    assert L.nb_reduce_dbias(P, P, 8, 12, 0) == binding.NB_ERR_UNSUPPORTED
+    assert L.nb_debug_wait_timeout(0) == binding.NB_ERR_INVALID_ARG
+    assert L.nb_workspace_reserve(-5) == binding.NB_ERR_INVALID_ARG
+
+
+def test_forward_with_zero_rows_is_a_no_op_everywhere(L):
+    P = 0x10000
+    assert L.nb_linear_forward_ex(P, None, P, P, None, 0, 8, 8, 0, None) == binding.NB_OK
+
+
+def test_binding_has_no_cpu_path(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError, match="missing"):
+        binding.lib()

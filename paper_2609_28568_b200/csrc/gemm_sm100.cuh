@@ -3,8 +3,9 @@
 //   warp 0      TMA producer: fills a ring of shared-memory stages (A tile 128x64, B tile Nx64)
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (128 x BLOCK_N x 16) into TMEM;
 //               two accumulators so the next tile's main loop overlaps this tile's epilogue
-//   warps 2..5  epilogue: tcgen05.ld -> fp32 registers -> bias / activation -> swizzled
-//               shared staging -> TMA store (or TMA reduce-add for split-K fp32 results)
+//   warps 2..9  epilogue: tcgen05.ld -> fp32 registers -> bias / activation -> swizzled
+//               shared staging -> TMA store (or TMA reduce-add for split-K fp32 results);
+//               two warps per TMEM lane quarter, each taking half of a step's columns
 //
 // Operand layouts. "K-major" means the reduction index is contiguous in global memory (forward:
 // both operands). "MN-major" means the output index is contiguous (dgrad reads the weight as
@@ -29,8 +30,9 @@ namespace nb {
 constexpr int kBlockM = 128;
 constexpr int kBlockK = 64;   // bf16 elements per stage along K = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kNumThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kNumThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int kEpiThreads = 256;
+constexpr int kEpiWarps = 8;
 constexpr uint32_t kStgBytes = 16384;  // one staging buffer: 128 rows x 128 bytes
 constexpr int kStatusTimeout = 4;      // == NB_ERR_TIMEOUT
 constexpr int kStatusBadSmem = 5;
@@ -223,7 +225,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
-            ptx::mbar_init(tempty_bar(b), 4 * CG);  // one arrive per epilogue warp of the tile
+            ptx::mbar_init(tempty_bar(b), kEpiWarps * CG);  // one arrive per epilogue warp of the tile
         }
         for (int b = 0; b < 4; ++b) ptx::mbar_init(aux_bar(b), 1);
         ptx::st_shared_u32_volatile(abort_addr, 0);
@@ -367,11 +369,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
-        const int q = warp & 3;           // TMEM lane quarter this warp may read
-        const int row = q * 32 + lane;    // row of the tile owned by this thread
+        // ------------------------------------------------------------ epilogue (warps 2..9)
+        // Warp w may read TMEM lanes 32*(w%4)..+31, i.e. rows q*32..q*32+31 of the tile. Two warps
+        // share each lane quarter and split every step's columns in halves (hf = 0 / 1).
+        const int q = warp & 3;
+        const int hf = (warp - 2) >> 2;
+        const int row = q * 32 + lane;
         const bool leader = (threadIdx.x == 64);
-        const int et = static_cast<int>(threadIdx.x) - 64;  // 0..127
+        const int et = static_cast<int>(threadIdx.x) - 64;  // 0..255
         const uint32_t stg0 = smem + Cfg::OFF_STG;
         const uint32_t bias_s = smem + Cfg::OFF_BIAS;
         const uint32_t row_off = static_cast<uint32_t>(row) * 128u;
@@ -397,17 +402,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t ab = aux_bar(static_cast<int>(slot));
             ptx::mbar_expect_tx(ab, kStgBytes);
             ptx::tma_load_2d(stg0 + slot * kStgBytes, &tmE, ab, x,
-                             m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM);
+                             ptx::fresh(m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM));
         };
         if (EPI == kEpiMulGeluGrad && leader) {
             for (uint32_t g = 0; g < AUX_AHEAD; ++g) issue_aux(g);
         }
+        __syncwarp();
 
         // the accumulator is handed back on the leader CTA's barrier
         auto release_acc = [&](int a) {
-            if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(a), 0));
-            else ptx::mbar_arrive(tempty_bar(a));
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(a), 0));
+                else ptx::mbar_arrive(tempty_bar(a));
+            }
+            __syncwarp();
         };
+        // 8 bf16 columns (one 16-byte chunk) of this thread's row in a staging buffer
+        auto chunk_pos = [&](int chunk) { return row_off + ((static_cast<uint32_t>(chunk) ^ sw) << 4); };
 
         for (int u = first_unit; u < num_units; u += unit_stride) {
             // uniform exit: the flag is only written by epilogue threads inside a unit, and
@@ -443,74 +456,64 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const uint32_t buf = stg0 + slot * Cfg::BUFS_PER_STEP * kStgBytes;
 
                 if (EPI == kEpiStore || EPI == kEpiGelu) {
-                    uint32_t r0[32], r1[32];
-                    ptx::tmem_ld_32x32_x2_wait(t_acc + c * 64, t_acc + c * 64 + 32, r0, r1);
-                    if (c == STEPS - 1) {  // accumulator fully read: hand it back to the MMA warp
-                        ptx::tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) release_acc(acc);
-                    }
+                    // this thread: columns [c*64 + hf*32, +32) of its row
+                    const int col0 = c * 64 + hf * 32;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32_wait(t_acc + col0, r);
+                    if (c == STEPS - 1) release_acc(acc);  // accumulator fully read
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            float v[8];
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const uint32_t bits = (h == 0) ? r0[j * 8 + k] : r1[j * 8 + k];
-                                v[k] = __uint_as_float(bits) +
-                                       ptx::ld_shared_f32(bias_s + 4u * (c * 64 + h * 32 + j * 8 + k));
-                            }
-                            const uint32_t pos = row_off + (((h * 4 + j) ^ sw) << 4);
-                            if (EPI == kEpiGelu) {
-                                ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(v[0], v[1]),
-                                                  ptx::pack_bf16x2(v[2], v[3]),
-                                                  ptx::pack_bf16x2(v[4], v[5]),
-                                                  ptx::pack_bf16x2(v[6], v[7]));
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) v[k] = gelu_fwd(v[k]);
-                            }
-                            ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(v[0], v[1]),
-                                              ptx::pack_bf16x2(v[2], v[3]),
-                                              ptx::pack_bf16x2(v[4], v[5]),
+                    for (int j = 0; j < 4; ++j) {
+                        float v[8];
+                        float4 b0, b1;
+                        ptx::ld_shared_f32x4(bias_s + 4u * (col0 + j * 8), b0);
+                        ptx::ld_shared_f32x4(bias_s + 4u * (col0 + j * 8 + 4), b1);
+                        v[0] = __uint_as_float(r[j * 8 + 0]) + b0.x;
+                        v[1] = __uint_as_float(r[j * 8 + 1]) + b0.y;
+                        v[2] = __uint_as_float(r[j * 8 + 2]) + b0.z;
+                        v[3] = __uint_as_float(r[j * 8 + 3]) + b0.w;
+                        v[4] = __uint_as_float(r[j * 8 + 4]) + b1.x;
+                        v[5] = __uint_as_float(r[j * 8 + 5]) + b1.y;
+                        v[6] = __uint_as_float(r[j * 8 + 6]) + b1.z;
+                        v[7] = __uint_as_float(r[j * 8 + 7]) + b1.w;
+                        const uint32_t pos = chunk_pos(hf * 4 + j);
+                        if (EPI == kEpiGelu) {
+                            ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(v[0], v[1]),
+                                              ptx::pack_bf16x2(v[2], v[3]), ptx::pack_bf16x2(v[4], v[5]),
                                               ptx::pack_bf16x2(v[6], v[7]));
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) v[k] = gelu_fwd(v[k]);
                         }
+                        ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(v[0], v[1]),
+                                          ptx::pack_bf16x2(v[2], v[3]), ptx::pack_bf16x2(v[4], v[5]),
+                                          ptx::pack_bf16x2(v[6], v[7]));
                     }
                 } else if (EPI == kEpiSwiglu) {
-                    // step c covers out columns [c*64, c*64+64): gate TMEM cols c*64.., up cols 128+c*64..
+                    // step c covers out columns [c*64, +64): gate TMEM cols c*64.., up cols 128 + c*64..
+                    const int col0 = c * 64 + hf * 32;
+                    uint32_t rg[32], ru[32];
+                    ptx::tmem_ld_32x32_x2_wait(t_acc + col0, t_acc + 128 + col0, rg, ru);
+                    if (c == STEPS - 1) release_acc(acc);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t rg[32], ru[32];
-                        ptx::tmem_ld_32x32_x2_wait(t_acc + c * 64 + h * 32, t_acc + 128 + c * 64 + h * 32,
-                                                   rg, ru);
-                        if (c == STEPS - 1 && h == 1) {
-                            ptx::tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) release_acc(acc);
+                    for (int j = 0; j < 4; ++j) {
+                        float g[8], uu[8], o[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const int cc = col0 + j * 8 + k;
+                            g[k] = __uint_as_float(rg[j * 8 + k]) + ptx::ld_shared_f32(bias_s + 4u * cc);
+                            uu[k] = __uint_as_float(ru[j * 8 + k]) +
+                                    ptx::ld_shared_f32(bias_s + 4u * (128 + cc));
+                            o[k] = silu_fwd(g[k]) * uu[k];
                         }
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            float g[8], uu[8], o[8];
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const int cc = c * 64 + h * 32 + j * 8 + k;
-                                g[k] = __uint_as_float(rg[j * 8 + k]) + ptx::ld_shared_f32(bias_s + 4u * cc);
-                                uu[k] = __uint_as_float(ru[j * 8 + k]) +
-                                        ptx::ld_shared_f32(bias_s + 4u * (128 + cc));
-                                o[k] = silu_fwd(g[k]) * uu[k];
-                            }
-                            const uint32_t pos = row_off + (((h * 4 + j) ^ sw) << 4);
-                            ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(o[0], o[1]),
-                                              ptx::pack_bf16x2(o[2], o[3]), ptx::pack_bf16x2(o[4], o[5]),
-                                              ptx::pack_bf16x2(o[6], o[7]));
-                            ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(g[0], g[1]),
-                                              ptx::pack_bf16x2(g[2], g[3]), ptx::pack_bf16x2(g[4], g[5]),
-                                              ptx::pack_bf16x2(g[6], g[7]));
-                            ptx::st_shared_v4(buf + 2 * kStgBytes + pos, ptx::pack_bf16x2(uu[0], uu[1]),
-                                              ptx::pack_bf16x2(uu[2], uu[3]),
-                                              ptx::pack_bf16x2(uu[4], uu[5]),
-                                              ptx::pack_bf16x2(uu[6], uu[7]));
-                        }
+                        const uint32_t pos = chunk_pos(hf * 4 + j);
+                        ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(o[0], o[1]),
+                                          ptx::pack_bf16x2(o[2], o[3]), ptx::pack_bf16x2(o[4], o[5]),
+                                          ptx::pack_bf16x2(o[6], o[7]));
+                        ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(g[0], g[1]),
+                                          ptx::pack_bf16x2(g[2], g[3]), ptx::pack_bf16x2(g[4], g[5]),
+                                          ptx::pack_bf16x2(g[6], g[7]));
+                        ptx::st_shared_v4(buf + 2 * kStgBytes + pos, ptx::pack_bf16x2(uu[0], uu[1]),
+                                          ptx::pack_bf16x2(uu[2], uu[3]), ptx::pack_bf16x2(uu[4], uu[5]),
+                                          ptx::pack_bf16x2(uu[6], uu[7]));
                     }
                 } else if (EPI == kEpiMulGeluGrad) {
                     bool aok = true;
@@ -518,45 +521,36 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         aok = wait_barrier(wctx, aux_bar(static_cast<int>(slot)), (gstep / SLOTS) & 1u,
                                            500 + static_cast<int>(slot));
                     aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
-                    if (!aok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
-                    uint32_t r0[32], r1[32];
-                    ptx::tmem_ld_32x32_x2_wait(t_acc + c * 64, t_acc + c * 64 + 32, r0, r1);
-                    if (c == STEPS - 1) {
-                        ptx::tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) release_acc(acc);
+                    if (!aok) {
+                        ptx::st_shared_u32_volatile(epi_abort_addr, 1);
+                        ok = false;
                     }
+                    const int col0 = c * 64 + hf * 32;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32_wait(t_acc + col0, r);
+                    if (c == STEPS - 1) release_acc(acc);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t pos = buf + chunk_pos(hf * 4 + j);
+                        uint32_t x[4];
+                        ptx::ld_shared_v4(pos, x[0], x[1], x[2], x[3]);
+                        uint32_t w[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t pos = buf + row_off + (((h * 4 + j) ^ sw) << 4);
-                            uint32_t x[4];
-                            ptx::ld_shared_v4(pos, x[0], x[1], x[2], x[3]);
-                            uint32_t w[4];
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const uint32_t b0 = (h == 0) ? r0[j * 8 + 2 * k] : r1[j * 8 + 2 * k];
-                                const uint32_t b1 = (h == 0) ? r0[j * 8 + 2 * k + 1] : r1[j * 8 + 2 * k + 1];
-                                const float lo = __uint_as_float(b0) * gelu_bwd(ptx::bf16_lo(x[k]));
-                                const float hi = __uint_as_float(b1) * gelu_bwd(ptx::bf16_hi(x[k]));
-                                w[k] = ptx::pack_bf16x2(lo, hi);
-                            }
-                            ptx::st_shared_v4(pos, w[0], w[1], w[2], w[3]);
+                        for (int k = 0; k < 4; ++k) {
+                            const float lo = __uint_as_float(r[j * 8 + 2 * k]) * gelu_bwd(ptx::bf16_lo(x[k]));
+                            const float hi = __uint_as_float(r[j * 8 + 2 * k + 1]) * gelu_bwd(ptx::bf16_hi(x[k]));
+                            w[k] = ptx::pack_bf16x2(lo, hi);
                         }
+                        ptx::st_shared_v4(pos, w[0], w[1], w[2], w[3]);
                     }
-                } else {  // kEpiF32: 32 fp32 columns per step
-                    uint32_t r0[32];
-                    ptx::tmem_ld_32x32_wait(t_acc + c * 32, r0);
-                    if (c == STEPS - 1) {
-                        ptx::tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) release_acc(acc);
-                    }
+                } else {  // kEpiF32: 32 fp32 columns per step, 16 per thread
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16_wait(t_acc + c * 32 + hf * 16, r);
+                    if (c == STEPS - 1) release_acc(acc);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        ptx::st_shared_v4(buf + row_off + ((j ^ sw) << 4), r0[j * 4], r0[j * 4 + 1],
-                                          r0[j * 4 + 2], r0[j * 4 + 3]);
+                    for (int j = 0; j < 4; ++j)
+                        ptx::st_shared_v4(buf + chunk_pos(hf * 4 + j), r[j * 4], r[j * 4 + 1],
+                                          r[j * 4 + 2], r[j * 4 + 3]);
                 }
 
                 // make the staged tile visible to the TMA engine, then one thread stores it

@@ -151,6 +151,40 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
 int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int accumulate);
 
 /*
+ * Bias gradient of a GELU layer without any allocation (the paper has no counterpart; this
+ * exists for callers that must not allocate device memory):
+ *
+ *     dbias[o] (+)= sum over rows m of  dout[m, o] * gelu'(pre_act[m, o])
+ *
+ * It computes what nb_linear_backward_ex computes for `dbias` when it is given `pre_act`
+ * and NB_ACT_GELU, but where that call keeps dz = dout * gelu'(pre_act) in a workspace it
+ * obtains with cudaMalloc, this one keeps dz in a fixed array compiled into the library
+ * image (NB_NOALLOC_MAX_ELEMS bf16 elements, 8 MiB, resident on every GPU that loads the
+ * library until the process exits). Who needs it: code that runs where cudaMalloc is
+ * forbidden or unsafe, for example between other libraries' timing-critical sections, in
+ * processes whose device memory is fully handed to another allocator, or inside a service
+ * that promised its host a fixed footprint.
+ *
+ *   dbias   [i/o] [OC] fp32, device, 16-byte aligned; overwritten when accumulate == 0
+ *   dout    [in]  [BT, OC] bf16, device, 16-byte aligned
+ *   pre_act [in]  [BT, OC] bf16, device, 16-byte aligned
+ *   stream        cudaStream_t as void*
+ * Limits and errors: OC a multiple of 8; BT*OC must not exceed NB_NOALLOC_MAX_ELEMS,
+ * otherwise NB_ERR_UNSUPPORTED with a message naming the limit (nothing is launched).
+ * The call uses no cudaMalloc / cudaFree and no allocating library routine. The first call
+ * on each device looks up the device address of the built-in array (one
+ * cudaGetSymbolAddress, with that device current); make that first call before starting any
+ * stream capture.
+ * The array is shared by every call on the device and keeps what the last call wrote. Each
+ * call overwrites the part it uses before reading it, so nothing has to start at zero; but
+ * two calls whose kernels may overlap on the GPU (different streams, no ordering between
+ * them) race on it and must be serialised by the caller.
+ */
+#define NB_NOALLOC_MAX_ELEMS 4194304
+int nb_gelu_dbias_noalloc(void *dbias, const void *dout, const void *pre_act, int64_t BT,
+                          int64_t OC, int accumulate, void *stream);
+
+/*
  * Make sure the workspace holds at least `bytes` (so later calls do not allocate), or
  * release everything the library holds on the current device (workspace, status word,
  * descriptor cache) with nb_release.

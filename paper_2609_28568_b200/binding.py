@@ -22,7 +22,7 @@ EXPORTS = (
     "nb_version", "nb_last_error", "nb_set_stream", "nb_get_stream", "nb_linear_out_elems",
     "nb_linear_forward", "nb_linear_forward_ex", "nb_linear_backward", "nb_linear_backward_ex",
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
-    "nb_debug_wait_timeout", "nb_kernel_launches",
+    "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
 )
 
 _lib = None
@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
         L.nb_workspace_reserve.argtypes = [_i64]
         L.nb_debug_wait_timeout.argtypes = [_i64]
         L.nb_kernel_launches.restype = _i64
+        L.nb_gelu_dbias_noalloc.argtypes = [_vp, _vp, _vp, _i64, _i64, _int, _vp]
         _lib = L
     return _lib
 
@@ -137,6 +138,16 @@ def nb_release() -> None:
 def nb_check_status() -> None:
     """Synchronise and raise NbError(NB_ERR_TIMEOUT / NB_ERR_CUDA) if a kernel reported a failure."""
     _check(lib().nb_check_status())
+
+
+NOALLOC_MAX_ELEMS = 4194304
+
+
+def nb_gelu_dbias_noalloc(dbias, dout, pre_act, BT, OC, accumulate, stream=None) -> None:
+    """dbias (+)= column sums of dout * gelu'(pre_act), using only the scratch array built into
+    the library: for callers that may not allocate device memory. BT*OC <= NOALLOC_MAX_ELEMS."""
+    _check(lib().nb_gelu_dbias_noalloc(_ptr(dbias), _ptr(dout), _ptr(pre_act), BT, OC,
+                                       int(accumulate), _stream() if stream is None else stream))
 
 
 def nb_kernel_launches() -> int:

@@ -610,4 +610,64 @@ int nb_debug_wait_timeout(int64_t limit_us)
     return NB_OK;
 }
 
+// ----------------------------------------------------------------------------- no allocation
+// Scratch for nb_gelu_dbias_noalloc: part of the library image, so it exists on every device that
+// loads the library without anyone allocating it. In host code `nb_noalloc_scratch` is only a
+// handle for the runtime, not a device address: the address a kernel can use comes from
+// cudaGetSymbolAddress, once per device.
+}  // extern "C" (the array and its bookkeeping have internal linkage)
+
+namespace {
+static __device__ __align__(256) unsigned char nb_noalloc_scratch[NB_NOALLOC_MAX_ELEMS * 2];
+void *g_noalloc_ptr[kMaxDevices] = {};
+int g_noalloc_sms[kMaxDevices] = {};
+}  // namespace
+
+extern "C" {
+
+int nb_gelu_dbias_noalloc(void *dbias, const void *dout, const void *pre_act, int64_t BT, int64_t OC,
+                          int accumulate, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!dbias || !dout || !pre_act)
+        return fail(NB_ERR_INVALID_ARG, "dbias, dout and pre_act must not be NULL");
+    if (BT < 0 || OC <= 0) return fail(NB_ERR_INVALID_ARG, "negative or zero dimension");
+    if (OC % 8 != 0) return fail(NB_ERR_UNSUPPORTED, "OC must be a multiple of 8");
+    if (!aligned16(dbias) || !aligned16(dout) || !aligned16(pre_act))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (BT >= (1ll << 31) || OC >= (1ll << 31) || BT * OC > static_cast<int64_t>(NB_NOALLOC_MAX_ELEMS))
+        return fail(NB_ERR_UNSUPPORTED,
+                    "BT*OC = %lld exceeds the built-in scratch of %d elements (NB_NOALLOC_MAX_ELEMS); "
+                    "use nb_linear_backward_ex, which allocates a workspace",
+                    static_cast<long long>(BT * OC), NB_NOALLOC_MAX_ELEMS);
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    int dev = 0;
+    NB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(NB_ERR_UNSUPPORTED, "device index %d", dev);
+    if (!g_noalloc_ptr[dev]) {  // set-up, once per device, with that device current
+        void *ptr = nullptr;
+        NB_CUDA(cudaGetSymbolAddress(&ptr, nb_noalloc_scratch));
+        int sms = 0;
+        NB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        if (!ptr || sms <= 0) return fail(NB_ERR_CUDA, "could not resolve the built-in scratch array");
+        g_noalloc_sms[dev] = sms;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    DeviceState local;  // only the SM count is read by the launch helpers below
+    local.num_sms = g_noalloc_sms[dev];
+    void *dz = g_noalloc_ptr[dev];
+
+    if (BT > 0) {
+        // dz = dout * gelu'(pre_act) overwrites the first BT*OC elements of the scratch
+        const long long nvec = BT * OC / 8;
+        gelu_backward_kernel<<<elementwise_grid(local, nvec), 256, 0, stream>>>(
+            static_cast<uint4 *>(dz), static_cast<const uint4 *>(dout),
+            static_cast<const uint4 *>(pre_act), nvec);
+        NB_CUDA(cudaGetLastError());
+        ++g_launches;
+    }
+    return launch_dbias(local, static_cast<float *>(dbias), dz, BT, OC, accumulate, stream);
+}
+
 }  // extern "C"

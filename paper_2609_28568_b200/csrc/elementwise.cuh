@@ -70,7 +70,7 @@ swiglu_backward_kernel(uint4 *__restrict__ dz, const uint4 *__restrict__ dout,
 // A block owns 128 columns and `rows_per_block` rows. Inside a warp, lanes 0..7 hold eight
 // 128-bit column vectors (64 columns) and the lane's upper bits select one of four rows, for two
 // 64-column halves; rows are summed in registers, then across the four row lanes by shuffles,
-// across the eight warps through shared memory, and across blocks by atomic adds.
+// across the eight warps by shared-memory atomics, and across blocks by global atomic adds.
 constexpr int kDbiasCols = 128;
 constexpr int kDbiasThreads = 256;
 
@@ -78,13 +78,15 @@ __global__ void __launch_bounds__(kDbiasThreads)
 dbias_kernel(float *__restrict__ dbias, const __nv_bfloat16 *__restrict__ dz, long long BT, int OC,
              int rows_per_block)
 {
-    __shared__ float part[8][kDbiasCols];
+    // 512 bytes of shared memory only: small enough to share an SM with a resident GEMM CTA
+    __shared__ float part[kDbiasCols];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cv = lane & 7;   // column vector inside a 64-column half
     const int rs = lane >> 3;  // row inside a group of four
     const int col0 = blockIdx.x * kDbiasCols;
     const long long r_begin = static_cast<long long>(blockIdx.y) * rows_per_block;
     const long long r_end = min(r_begin + rows_per_block, BT);
+    if (threadIdx.x < kDbiasCols) part[threadIdx.x] = 0.0f;
     float acc[2][8];
 #pragma unroll
     for (int h = 0; h < 2; ++h)
@@ -107,6 +109,7 @@ dbias_kernel(float *__restrict__ dbias, const __nv_bfloat16 *__restrict__ dz, lo
             acc[1][2 * k + 1] += ptx::bf16_hi(b[k]);
         }
     }
+    __syncthreads();
 #pragma unroll
     for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -114,15 +117,12 @@ dbias_kernel(float *__restrict__ dbias, const __nv_bfloat16 *__restrict__ dz, lo
             float v = acc[h][k];
             v += __shfl_xor_sync(0xffffffffu, v, 8);
             v += __shfl_xor_sync(0xffffffffu, v, 16);
-            if (rs == 0) part[warp][h * 64 + cv * 8 + k] = v;
+            if (rs == 0) atomicAdd(&part[h * 64 + cv * 8 + k], v);
         }
     __syncthreads();
     if (threadIdx.x < kDbiasCols) {
-        float s = 0.0f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
         const int col = col0 + threadIdx.x;
-        if (col < OC) atomicAdd(dbias + col, s);
+        if (col < OC) atomicAdd(dbias + col, part[threadIdx.x]);
     }
 }
 

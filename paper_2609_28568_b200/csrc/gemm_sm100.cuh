@@ -7,6 +7,8 @@
 //               shared staging -> TMA store (or TMA reduce-add for split-K fp32 results);
 //               two warps per TMEM lane quarter, each taking half of a step's columns
 //
+//   warps 10..13 (wgrad with fused bias gradient only) sum the A tiles over k from shared memory
+//
 // Operand layouts. "K-major" means the reduction index is contiguous in global memory (forward:
 // both operands). "MN-major" means the output index is contiguous (dgrad reads the weight as
 // B[n=c, k=o] from W[o, c]; wgrad reads dz and inp as A[m=o, k=row], B[n=c, k=row]); those tiles
@@ -55,12 +57,18 @@ struct GemmParams {
     int swiglu_h;           // kEpiSwiglu: H (gate rows [0,H), up rows [H,2H) of B)
     int reduce;             // kEpiF32: 1 reduce-add into D, 0 overwrite
     const __nv_bfloat16 *bias;  // [N] or nullptr
+    float *dbias;               // wgrad with fused bias gradient: dbias[m] += sum_k A[m,k]
     int *status;
     unsigned long long timeout_ns;
 };
 
-template <int CG_, int BLOCK_N_, int STAGES_, int NSTG_, bool A_MN_, bool B_MN_, int EPI_>
+template <int CG_, int BLOCK_N_, int STAGES_, int NSTG_, bool A_MN_, bool B_MN_, int EPI_,
+          bool DBIAS_ = false>
 struct GemmCfg {
+    // DBIAS: four extra warps sum the A tiles (dz^T in wgrad) over k while the tensor core reads
+    // them, so the bias gradient needs no pass of its own over dz
+    static constexpr bool DBIAS = DBIAS_;
+    static constexpr int THREADS = kNumThreads + (DBIAS_ ? 128 : 0);
     static constexpr int CG = CG_;              // CTAs per tile: 1, or 2 (a cta_group::2 pair)
     static constexpr int TILE_M = kBlockM * CG_;
     static constexpr int BLOCK_N = BLOCK_N_;
@@ -94,6 +102,7 @@ struct GemmCfg {
     static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 3, "aux prefetch needs a ring of >= 3");
     static_assert(EPI != kEpiSwiglu || BLOCK_N == 256, "SwiGLU tiles pair 128 gate + 128 up cols");
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+    static_assert(!DBIAS_ || (A_MN_ && EPI_ == kEpiF32), "the fused bias gradient belongs to wgrad");
 };
 
 // barrier slots inside the 256-byte barrier region (8 bytes each)
@@ -182,8 +191,13 @@ __device__ __forceinline__ float gelu_bwd(float x)
 }
 __device__ __forceinline__ float silu_fwd(float g) { return __fdividef(g, 1.0f + __expf(-g)); }
 
+__device__ __forceinline__ void atomicAdd_shared_f32(uint32_t addr, float v)
+{
+    asm volatile("red.shared.add.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
 template <class Cfg>
-__global__ void __launch_bounds__(kNumThreads, 1)
+__global__ void __launch_bounds__(Cfg::THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmE,
             const GemmParams p)
@@ -213,15 +227,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
     auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
     auto aux_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 4 + b); };
+    // DBIAS only: a stage is handed MMA -> reducers (empty_bar) -> producer (free_bar)
+    auto free_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 8 + s); };
     const uint32_t tmem_slot = bar0 + 240;
     const uint32_t abort_addr = bar0 + 244;
     const uint32_t epi_abort_addr = bar0 + 248;
-    static_assert(8 * (2 * STAGES + 8) <= 240, "barrier region");
+    static_assert(8 * (3 * STAGES + 8) <= 240, "barrier region");
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(full_bar(s), 1);
-            ptx::mbar_init(empty_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);  // MMAs that read the stage are done
+            ptx::mbar_init(free_bar(s), 4);   // DBIAS: the four reducer warps have read it too
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(tfull_bar(b), 1);
@@ -270,7 +287,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const int kb1 = min(kb0 + p.kblocks_per_split, p.kblocks);
                 const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    ok = wait_barrier(wctx, empty_bar(stage), phase ^ 1u, 100 + stage);
+                    ok = wait_barrier(wctx, Cfg::DBIAS ? free_bar(stage) : empty_bar(stage), phase ^ 1u,
+                                      100 + stage);
                     if (!ok) break;
                     // the leader's barrier collects the bytes of both CTAs of a pair
                     const uint32_t fb = (CG == 2) ? ptx::mapa(full_bar(stage), 0) : full_bar(stage);
@@ -366,6 +384,71 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     acc = 0;
                     acc_phase ^= 1u;
                 }
+            }
+        }
+    } else if (Cfg::DBIAS && warp >= 10) {
+        // ------------------------------------------------------------ bias-gradient reducers (warps 10..13)
+        // They read a stage after the tensor core has, and only then is it handed back to the
+        // producer. A tile of a stage (MN-major): two boxes of 64 k-rows x 128 bytes (64 m values), swizzled.
+        // Thread t sums chunk (t & 15) (8 consecutive m) over k rows (t >> 4) + 8 i. Only the units
+        // of the first n-tile do the arithmetic; every unit takes part in the stage hand-shake.
+        const int rt = static_cast<int>(threadIdx.x) - 320;  // 0..127
+        const int cc = rt & 15;
+        const int kbase = rt >> 4;
+        const uint32_t part_s = smem + Cfg::OFF_BIAS;  // 128 floats, unused by the fp32 epilogue
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        if (rt < kBlockM) ptx::st_shared_f32(part_s + 4u * rt, 0.0f);
+        ptx::named_bar_sync(2, 128);
+        for (int u = first_unit; u < num_units; u += unit_stride) {
+            int m_blk, n_blk, split;
+            decode_unit(p, u, m_blk, n_blk, split);
+            const int kb0 = split * p.kblocks_per_split;
+            const int kb1 = min(kb0 + p.kblocks_per_split, p.kblocks);
+            const bool mine = (n_blk == 0) && p.dbias != nullptr;
+            float sum[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) sum[k] = 0.0f;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (ok) {
+                    // wait until the tensor core is done with the stage: its completion is multicast
+                    // to both CTAs of a pair, so no CTA has to watch the other's barriers, and the
+                    // tile is still intact because the producer waits for the reducers
+                    bool w = true;
+                    if (lane == 0) w = wait_barrier(wctx, empty_bar(stage), phase, 600 + stage);
+                    ok = __shfl_sync(0xffffffffu, w ? 1 : 0, 0) != 0;
+                }
+                if (ok && mine) {
+                    const uint32_t sa = smem + Cfg::OFF_A + stage * Cfg::A_BYTES +
+                                        static_cast<uint32_t>(cc >> 3) * 8192u;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint32_t kr = static_cast<uint32_t>(kbase + 8 * i);
+                        uint32_t x[4];
+                        ptx::ld_shared_v4(sa + kr * 128u + (((cc & 7u) ^ (kr & 7u)) << 4), x[0], x[1], x[2], x[3]);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            sum[2 * k] += ptx::bf16_lo(x[k]);
+                            sum[2 * k + 1] += ptx::bf16_hi(x[k]);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(free_bar(stage));  // this warp is done with the stage
+                if (++stage == STAGES) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+            if (mine) {  // uniform across the four warps: same unit, same parameters
+#pragma unroll
+                for (int k = 0; k < 8; ++k) atomicAdd_shared_f32(part_s + 4u * (cc * 8 + k), sum[k]);
+                ptx::named_bar_sync(2, 128);
+                const int m = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM + rt;
+                if (ok && rt < kBlockM && m < p.M) atomicAdd(p.dbias + m, ptx::ld_shared_f32(part_s + 4u * rt));
+                if (rt < kBlockM) ptx::st_shared_f32(part_s + 4u * rt, 0.0f);
+                ptx::named_bar_sync(2, 128);
             }
         }
     } else {

@@ -177,6 +177,7 @@ struct GemmArgs {
     int swiglu_h;
     int reduce;
     int splits;
+    float *dbias;  // wgrad: bias gradient fused into the pass over dz, or null
 };
 
 template <class Cfg>
@@ -193,7 +194,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
         if (Cfg::CG == 2) {  // how many CTA pairs can be resident at once
             cudaLaunchConfig_t qc = {};
             qc.gridDim = dim3(static_cast<unsigned>(s.num_sms));
-            qc.blockDim = dim3(kNumThreads);
+            qc.blockDim = dim3(Cfg::THREADS);
             qc.dynamicSmemBytes = Cfg::SMEM_BYTES;
             cudaLaunchAttribute qa[1];
             qa[0].id = cudaLaunchAttributeClusterDimension;
@@ -238,6 +239,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     p.swiglu_h = a.swiglu_h;
     p.reduce = a.reduce;
     p.bias = static_cast<const __nv_bfloat16 *>(a.bias);
+    p.dbias = a.dbias;
     p.status = s.status;
     p.timeout_ns = kDefaultTimeoutNs;
     const long long units = 1ll * p.tiles_m * p.tiles_n * p.splits;
@@ -246,7 +248,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(clusters * Cfg::CG));
-    cfg.blockDim = dim3(kNumThreads);
+    cfg.blockDim = dim3(Cfg::THREADS);
     cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attrs[1];
@@ -277,6 +279,8 @@ using FwdSwiglu2 = GemmCfg<2, 256, 5, 3, false, false, kEpiSwiglu>;
 using DgradStore2 = GemmCfg<2, 256, 6, 2, false, true, kEpiStore>;
 using DgradMulGelu2 = GemmCfg<2, 256, 5, 4, false, true, kEpiMulGeluGrad>;
 using WgradF32_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32>;
+using WgradF32Bias1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32, true>;
+using WgradF32Bias2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32, true>;
 using WgradBf16_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiStore>;
 
 bool use_pairs(int M)
@@ -513,7 +517,14 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
             a.reduce = (accumulate || splits > 1) ? 1 : 0;
             if (!accumulate && splits > 1)
                 NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(OC * C) * 4, stream));
-            rc = launch_gemm_auto<WgradF32_1, WgradF32_2>(*s, a, stream);
+            if (dbias) {  // the bias gradient rides along: reducer warps sum dz while it is in shared memory
+                if (!accumulate) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
+                a.dbias = static_cast<float *>(dbias);
+                rc = launch_gemm_auto<WgradF32Bias1, WgradF32Bias2>(*s, a, stream);
+                dbias = nullptr;  // done
+            } else {
+                rc = launch_gemm_auto<WgradF32_1, WgradF32_2>(*s, a, stream);
+            }
         } else {
             a.d_dtype = 0;
             a.splits = 1;

@@ -228,17 +228,17 @@ def main():
         stack.step()
     nb.nb_check_status()
 
-    # ---- timed region: K steps, one event pair around the region and one around every call
-    records = []  # (kind, layer name, start event, end event)
+    # ---- timed region: K steps between two events on the launch stream. No events between the
+    # calls: an event record between two kernels keeps the second kernel's set-up from overlapping
+    # the first kernel's tail (programmatic dependent launch) and costs 2-3 % of the step.
+    records = []  # (kind, layer name, start event, end event), filled by the breakdown pass
 
     def hook(kind, L, begin):
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
         if begin:
-            e = torch.cuda.Event(enable_timing=True)
-            e.record()
             records.append([kind, L.spec.name, e, None])
         else:
-            e = torch.cuda.Event(enable_timing=True)
-            e.record()
             records[-1][3] = e
 
     props = torch.cuda.get_device_properties(dev)
@@ -250,11 +250,10 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.steps):
-        stack.step(hook)
+        stack.step()
     ev1.record()
     barrier()
     launches = nb.nb_kernel_launches() - launches0
-    clocks = sampler.stop()
     nb.nb_check_status()
     elapsed_ms = ev0.elapsed_time(ev1)
     if dist is not None:
@@ -264,6 +263,17 @@ def main():
     ms_per_step = elapsed_ms / args.steps
     tflops = world * flops_step / (ms_per_step * 1e-3) / 1e12
     tokens_per_s = world * tokens_step / (ms_per_step * 1e-3)
+
+    # ---- breakdown pass: the same K steps again, now with an event pair around every call
+    bev0, bev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    bev0.record()
+    for _ in range(args.steps):
+        stack.step(hook)
+    bev1.record()
+    barrier()
+    clocks = sampler.stop()
+    nb.nb_check_status()
+    breakdown_ms_per_step = bev0.elapsed_time(bev1) / args.steps
 
     # ---- per-call breakdown from the events of the timed region
     per = {}
@@ -296,7 +306,9 @@ def main():
         "bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
         "frac": achieved_tf / peak_tf, "traffic": traffic,
         "peak_source": f"{peak_src} cuBLAS bf16 ({'sustained' if long_step else 'burst'})",
-        "kernel": "nb::gemm_kernel (tcgen05 fwd / dgrad / wgrad instantiations), all launches of the timed region",
+        "kernel": "nb::gemm_kernel (tcgen05 fwd / dgrad / wgrad instantiations), all launches of a step; "
+                  "durations from a second pass over the same steps with events around every call",
+        "breakdown_pass_ms_per_step": breakdown_ms_per_step,
         "frac_of_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
         "per_call": breakdown,
     }

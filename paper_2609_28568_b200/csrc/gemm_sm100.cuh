@@ -189,6 +189,47 @@ __device__ __forceinline__ float gelu_bwd(float x)
     const float du = 0.7978845608028654f * (1.0f + 3.0f * 0.044715f * x2);
     return 0.5f * (1.0f + t) + 0.5f * x * (1.0f - t * t) * du;
 }
+// The same two functions on pairs (packed fp32): tanh-GELU of z, and acc * gelu'(x).
+__device__ __forceinline__ ptx::f2 gelu_fwd2(ptx::f2 z)
+{
+    const ptx::f2 c0 = ptx::make_f2(0.7978845608028654f, 0.7978845608028654f);
+    const ptx::f2 c01 = ptx::make_f2(0.7978845608028654f * 0.044715f, 0.7978845608028654f * 0.044715f);
+    const ptx::f2 half = ptx::make_f2(0.5f, 0.5f);
+    const ptx::f2 z2 = ptx::mul2(z, z);
+    const ptx::f2 u = ptx::mul2(z, ptx::fma2(z2, c01, c0));
+    float u0, u1;
+    ptx::split_f2(u, u0, u1);
+    const ptx::f2 t = ptx::make_f2(ptx::tanh_approx(u0), ptx::tanh_approx(u1));
+    const ptx::f2 hz = ptx::mul2(z, half);
+    return ptx::fma2(hz, t, hz);
+}
+__device__ __forceinline__ ptx::f2 mul_gelu_bwd2(ptx::f2 acc, ptx::f2 x)
+{
+    const ptx::f2 c0 = ptx::make_f2(0.7978845608028654f, 0.7978845608028654f);
+    const ptx::f2 c01 = ptx::make_f2(0.7978845608028654f * 0.044715f, 0.7978845608028654f * 0.044715f);
+    const ptx::f2 c03 = ptx::make_f2(3.0f * 0.7978845608028654f * 0.044715f,
+                                     3.0f * 0.7978845608028654f * 0.044715f);
+    const ptx::f2 half = ptx::make_f2(0.5f, 0.5f);
+    const ptx::f2 one = ptx::make_f2(1.0f, 1.0f);
+    const ptx::f2 neg1 = ptx::make_f2(-1.0f, -1.0f);
+    const ptx::f2 x2 = ptx::mul2(x, x);
+    const ptx::f2 u = ptx::mul2(x, ptx::fma2(x2, c01, c0));
+    float u0, u1;
+    ptx::split_f2(u, u0, u1);
+    const ptx::f2 t = ptx::make_f2(ptx::tanh_approx(u0), ptx::tanh_approx(u1));
+    const ptx::f2 du = ptx::fma2(x2, c03, c0);                    // d/dx of the tanh argument
+    const ptx::f2 a = ptx::fma2(t, half, half);                   // 0.5 (1 + t)
+    const ptx::f2 omt2 = ptx::fma2(ptx::mul2(t, t), neg1, one);   // 1 - t^2
+    const ptx::f2 b = ptx::mul2(ptx::mul2(x, half), du);          // 0.5 x du
+    return ptx::mul2(acc, ptx::fma2(b, omt2, a));
+}
+__device__ __forceinline__ uint32_t pack_f2_bf16x2(ptx::f2 v)
+{
+    float lo, hi;
+    ptx::split_f2(v, lo, hi);
+    return ptx::pack_bf16x2(lo, hi);
+}
+
 __device__ __forceinline__ float silu_fwd(float g) { return __fdividef(g, 1.0f + __expf(-g)); }
 
 __device__ __forceinline__ void atomicAdd_shared_f32(uint32_t addr, float v)
@@ -261,6 +302,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (CG == 2) ptx::cluster_sync();  // the peer's barriers are initialised before anyone signals them
     else __syncthreads();
     ptx::tc_fence_after();
+    // Everything above touched only this CTA's shared memory and TMEM, so it may run while the
+    // previous kernel of the stream is still draining; global memory is not read or written before
+    // that kernel has completed.
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
     const uint32_t tmem_base = ptx::ld_shared_u32_volatile(tmem_slot);
 
     const WaitCtx wctx{abort_addr, p.status, p.timeout_ns};
@@ -546,29 +592,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     if (c == STEPS - 1) release_acc(acc);  // accumulator fully read
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        float v[8];
                         float4 b0, b1;
                         ptx::ld_shared_f32x4(bias_s + 4u * (col0 + j * 8), b0);
                         ptx::ld_shared_f32x4(bias_s + 4u * (col0 + j * 8 + 4), b1);
-                        v[0] = __uint_as_float(r[j * 8 + 0]) + b0.x;
-                        v[1] = __uint_as_float(r[j * 8 + 1]) + b0.y;
-                        v[2] = __uint_as_float(r[j * 8 + 2]) + b0.z;
-                        v[3] = __uint_as_float(r[j * 8 + 3]) + b0.w;
-                        v[4] = __uint_as_float(r[j * 8 + 4]) + b1.x;
-                        v[5] = __uint_as_float(r[j * 8 + 5]) + b1.y;
-                        v[6] = __uint_as_float(r[j * 8 + 6]) + b1.z;
-                        v[7] = __uint_as_float(r[j * 8 + 7]) + b1.w;
+                        ptx::f2 z[4];  // eight columns as four packed pairs
+                        z[0] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 0], r[j * 8 + 1]), ptx::make_f2(b0.x, b0.y));
+                        z[1] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 2], r[j * 8 + 3]), ptx::make_f2(b0.z, b0.w));
+                        z[2] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 4], r[j * 8 + 5]), ptx::make_f2(b1.x, b1.y));
+                        z[3] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 6], r[j * 8 + 7]), ptx::make_f2(b1.z, b1.w));
                         const uint32_t pos = chunk_pos(hf * 4 + j);
                         if (EPI == kEpiGelu) {
-                            ptx::st_shared_v4(buf + kStgBytes + pos, ptx::pack_bf16x2(v[0], v[1]),
-                                              ptx::pack_bf16x2(v[2], v[3]), ptx::pack_bf16x2(v[4], v[5]),
-                                              ptx::pack_bf16x2(v[6], v[7]));
+                            ptx::st_shared_v4(buf + kStgBytes + pos, pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),
+                                              pack_f2_bf16x2(z[2]), pack_f2_bf16x2(z[3]));
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) v[k] = gelu_fwd(v[k]);
+                            for (int k = 0; k < 4; ++k) z[k] = gelu_fwd2(z[k]);
                         }
-                        ptx::st_shared_v4(buf + pos, ptx::pack_bf16x2(v[0], v[1]),
-                                          ptx::pack_bf16x2(v[2], v[3]), ptx::pack_bf16x2(v[4], v[5]),
-                                          ptx::pack_bf16x2(v[6], v[7]));
+                        ptx::st_shared_v4(buf + pos, pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),
+                                          pack_f2_bf16x2(z[2]), pack_f2_bf16x2(z[3]));
                     }
                 } else if (EPI == kEpiSwiglu) {
                     // step c covers out columns [c*64, +64): gate TMEM cols c*64.., up cols 128 + c*64..
@@ -620,9 +660,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         uint32_t w[4];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            const float lo = __uint_as_float(r[j * 8 + 2 * k]) * gelu_bwd(ptx::bf16_lo(x[k]));
-                            const float hi = __uint_as_float(r[j * 8 + 2 * k + 1]) * gelu_bwd(ptx::bf16_hi(x[k]));
-                            w[k] = ptx::pack_bf16x2(lo, hi);
+                            const ptx::f2 a2 = ptx::make_f2_bits(r[j * 8 + 2 * k], r[j * 8 + 2 * k + 1]);
+                            const ptx::f2 x2 = ptx::make_f2_bits(x[k] << 16, x[k] & 0xffff0000u);
+                            w[k] = pack_f2_bf16x2(mul_gelu_bwd2(a2, x2));
                         }
                         ptx::st_shared_v4(pos, w[0], w[1], w[2], w[3]);
                     }

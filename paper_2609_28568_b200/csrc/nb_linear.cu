@@ -25,6 +25,10 @@ constexpr int kMaxDevices = 64;
 constexpr unsigned long long kDefaultTimeoutNs = 2000000000ull;  // 2 s per wait
 
 std::atomic<long long> g_launches{0};
+const bool g_use_pdl = [] {
+    const char *e = getenv("NB_PDL");  // debugging aid: NB_PDL=0 turns dependent launch off
+    return !(e && e[0] == '0');
+}();
 thread_local std::string g_err;
 thread_local cudaStream_t g_stream = nullptr;
 
@@ -251,13 +255,17 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     cfg.blockDim = dim3(Cfg::THREADS);
     cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
     cfg.stream = stream;
-    cudaLaunchAttribute attrs[1];
+    cudaLaunchAttribute attrs[2];
     attrs[0].id = cudaLaunchAttributeClusterDimension;
     attrs[0].val.clusterDim.x = Cfg::CG;
     attrs[0].val.clusterDim.y = 1;
     attrs[0].val.clusterDim.z = 1;
+    // programmatic dependent launch: the kernel's set-up overlaps the previous kernel's tail; the
+    // kernel itself waits for that kernel before it touches global memory
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = g_use_pdl ? 2 : 1;
     NB_CUDA(cudaLaunchKernelEx(&cfg, gemm_kernel<Cfg>, tA, tB, tD, tE, p));
     ++g_launches;
     return NB_OK;

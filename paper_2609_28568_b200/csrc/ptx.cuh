@@ -29,6 +29,18 @@ __device__ __forceinline__ bool elect_one()
     return pred != 0;
 }
 
+// ------------------------------------------------------------------ programmatic dependent launch
+// launch_dependents: the next kernel of the stream may be scheduled as this grid's CTAs retire.
+// wait: block until every earlier grid has finished and its memory is visible.
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ------------------------------------------------------------------ clusters (CTA pairs)
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
@@ -312,6 +324,47 @@ __device__ __forceinline__ int fresh(int v)
 {
     asm volatile("mov.b32 %0, %0;" : "+r"(v));
     return v;
+}
+
+// ------------------------------------------------------------------ packed fp32 math (two lanes)
+// sm_100 executes fma / mul / add on pairs of fp32 held in a 64-bit register: half the issue slots
+// of the scalar forms, which is what the activation epilogues are short of.
+struct f2 {
+    uint64_t v;
+};
+__device__ __forceinline__ f2 make_f2(float lo, float hi)
+{
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f2 make_f2_bits(uint32_t lo, uint32_t hi)
+{
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r.v) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void split_f2(f2 a, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a.v));
+}
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c)
+{
+    f2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v));
+    return r;
+}
+__device__ __forceinline__ f2 mul2(f2 a, f2 b)
+{
+    f2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+    return r;
+}
+__device__ __forceinline__ f2 add2(f2 a, f2 b)
+{
+    f2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v));
+    return r;
 }
 
 // ------------------------------------------------------------------ math

@@ -118,11 +118,11 @@ def oracle_sample(seconds_hint: float = 15.0):
     import oracle
     from paper_2609_28568_b200 import shapes, synth
 
-    BT = 4096
+    BT = 8192
     specs = shapes.gpt2_block() + [shapes.gpt2_lm_head()]
     flops, secs = 0, 0.0
     for li, s in enumerate(specs):
-        rows = BT if s.OC != shapes.VOCAB_PADDED else 512
+        rows = BT if s.OC != shapes.VOCAB_PADDED else 1024
         f = lambda t: t.float().numpy()
         inp = f(synth.normal(9000 + li, (rows, s.C), 1.0))
         w = f(synth.normal(9100 + li, (s.OC, s.C), s.w_std))
@@ -135,7 +135,7 @@ def oracle_sample(seconds_hint: float = 15.0):
         secs += time.perf_counter() - t0
         flops += 6 * rows * s.C * s.OC
     desc = (f"fp32 oracle on one GPT-2 block (qkv, attn-proj, fc+GELU, proj) fwd+bwd at BT={BT} and the "
-            f"tied head fwd+bwd on 512 rows; {flops / 1e9:.1f} GFLOP")
+            f"tied head fwd+bwd on 1024 rows; {flops / 1e9:.1f} GFLOP")
     return flops, secs, desc, oracle.num_threads()
 
 
@@ -292,7 +292,9 @@ def main():
         gemm_flops += fl * n
         gemm_ms += ms
     peaks, peak_src = load_peaks()
-    long_step = ms_per_step * args.steps > 1000.0
+    # the GPU is under load for warm-up + timed + breakdown steps back to back: over a second of
+    # that is the "kernel timed inside a long step" case, judged against the sustained peak
+    long_step = ms_per_step * (args.warmup + 2 * args.steps) > 1000.0
     peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
     achieved_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     traffic = None
@@ -310,6 +312,8 @@ def main():
                   "durations from a second pass over the same steps with events around every call",
         "breakdown_pass_ms_per_step": breakdown_ms_per_step,
         "frac_of_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
+        "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
+        "frac_of_sustained_peak": achieved_tf / peaks["bf16_tflops_sustained"],
         "per_call": breakdown,
     }
 

@@ -206,6 +206,15 @@ int nb_check_status(void);
 int64_t nb_kernel_launches(void);
 
 /*
+ * Host-only view of how a wgrad of shape dweight[M, N] = sum over K rows is cut into work units
+ * (no device is touched): out[0] = row tiles, out[1] = column tiles, out[2] = split-K factor,
+ * out[3] = 64-row k-blocks per split, out[4] = k-blocks in total. `tile_m` is 128 or 256 (CTA
+ * pair), `slots` the number of tiles resident at once (SMs, or SM pairs). Unit u covers k-blocks
+ * [s*out[3], min((s+1)*out[3], out[4])) of tile t, with s = u / (out[0]*out[1]), t = u % (...).
+ */
+int nb_debug_split_plan(int64_t M, int64_t N, int64_t K, int slots, int tile_m, int *out);
+
+/*
  * Self-test of the bounded-wait mechanism: launches a one-block kernel that waits, for
  * at most `limit_us` microseconds, on a barrier nothing ever signals, then returns
  * normally after recording the expiry. nb_check_status() afterwards reports

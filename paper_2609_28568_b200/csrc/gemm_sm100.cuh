@@ -83,7 +83,11 @@ struct GemmCfg {
     static constexpr uint32_t OFF_A = 0;
     static constexpr uint32_t OFF_B = STAGES * A_BYTES;
     static constexpr uint32_t OFF_STG = STAGES * (A_BYTES + B_BYTES);
-    static constexpr uint32_t OFF_BIAS = OFF_STG + NSTG * kStgBytes;
+    // kEpiMulGeluGrad: a ring of NAUX buffers receives the pre-activation tiles, apart from the
+    // staging buffers, so the prefetch never waits for a store to drain
+    static constexpr int NAUX = (EPI_ == kEpiMulGeluGrad) ? 4 : 0;
+    static constexpr uint32_t OFF_AUX = OFF_STG + NSTG * kStgBytes;
+    static constexpr uint32_t OFF_BIAS = OFF_AUX + NAUX * kStgBytes;
     static constexpr uint32_t OFF_BAR = OFF_BIAS + BLOCK_N * 4;
     static constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
     static constexpr uint32_t TMEM_COLS = (2 * BLOCK_N <= 32) ? 32
@@ -99,7 +103,7 @@ struct GemmCfg {
     static_assert(BLOCK_N % (64 * CG_) == 0 && BLOCK_N >= 64 && BLOCK_N <= 256, "BLOCK_N");
     static_assert(2 * BLOCK_N <= 512, "two accumulators must fit in TMEM");
     static_assert(NSTG % BUFS_PER_STEP == 0 && SLOTS >= 1, "staging ring");
-    static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 3, "aux prefetch needs a ring of >= 3");
+    static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 2, "staging ring");
     static_assert(EPI != kEpiSwiglu || BLOCK_N == 256, "SwiGLU tiles pair 128 gate + 128 up cols");
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
     static_assert(!DBIAS_ || (A_MN_ && EPI_ == kEpiF32), "the fused bias gradient belongs to wgrad");
@@ -110,7 +114,7 @@ struct GemmCfg {
 //   [S, 2S)     empty[s]    MMA -> TMA
 //   2S, 2S+1    tmem_full   MMA -> epilogue
 //   2S+2, 2S+3  tmem_empty  epilogue -> MMA
-//   2S+4 .. +7  aux_full    TMA -> epilogue (kEpiMulGeluGrad)
+//   2S+4 .. +7  aux_full    TMA -> epilogue (kEpiMulGeluGrad), one per buffer of the aux ring
 //   byte 240: TMEM base address, 244: abort flag (any role), 248: epilogue abort flag
 
 struct WaitCtx {
@@ -515,7 +519,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint32_t gstep = 0;  // epilogue steps done so far (drives the staging ring)
         constexpr int SLOTS = Cfg::SLOTS;
         constexpr int STEPS = Cfg::STEPS;
-        constexpr int AUX_AHEAD = 2;
+        constexpr int AUX_AHEAD = Cfg::NAUX;  // steps the pre-activation prefetch runs ahead
 
         // coordinates of the aux tile for global step g (kEpiMulGeluGrad)
         auto issue_aux = [&](uint32_t g) {
@@ -527,14 +531,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             int m_blk, n_blk, split;
             decode_unit(p, static_cast<int>(u), m_blk, n_blk, split);
             const int x = n_blk * BLOCK_N + c * 64;
-            const uint32_t slot = g % SLOTS;
+            const uint32_t slot = g % (Cfg::NAUX > 0 ? Cfg::NAUX : 1);
             const uint32_t ab = aux_bar(static_cast<int>(slot));
             ptx::mbar_expect_tx(ab, kStgBytes);
-            ptx::tma_load_2d(stg0 + slot * kStgBytes, &tmE, ab, x,
+            ptx::tma_load_2d(smem + Cfg::OFF_AUX + slot * kStgBytes, &tmE, ab, x,
                              ptx::fresh(m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM));
         };
-        if (EPI == kEpiMulGeluGrad && leader) {
-            for (uint32_t g = 0; g < AUX_AHEAD; ++g) issue_aux(g);
+        if constexpr (EPI == kEpiMulGeluGrad) {
+            if (leader) {
+                for (int g = 0; g < AUX_AHEAD; ++g) issue_aux(static_cast<uint32_t>(g));
+            }
         }
         __syncwarp();
 
@@ -639,10 +645,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                           ptx::pack_bf16x2(uu[6], uu[7]));
                     }
                 } else if (EPI == kEpiMulGeluGrad) {
+                    constexpr uint32_t NAUX = Cfg::NAUX > 0 ? Cfg::NAUX : 1;
+                    const uint32_t aslot = gstep % NAUX;
+                    const uint32_t abuf = smem + Cfg::OFF_AUX + aslot * kStgBytes;
                     bool aok = true;
                     if (lane == 0)
-                        aok = wait_barrier(wctx, aux_bar(static_cast<int>(slot)), (gstep / SLOTS) & 1u,
-                                           500 + static_cast<int>(slot));
+                        aok = wait_barrier(wctx, aux_bar(static_cast<int>(aslot)), (gstep / NAUX) & 1u,
+                                           500 + static_cast<int>(aslot));
                     aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
                     if (!aok) {
                         ptx::st_shared_u32_volatile(epi_abort_addr, 1);
@@ -654,9 +663,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     if (c == STEPS - 1) release_acc(acc);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t pos = buf + chunk_pos(hf * 4 + j);
+                        const uint32_t cp = chunk_pos(hf * 4 + j);
                         uint32_t x[4];
-                        ptx::ld_shared_v4(pos, x[0], x[1], x[2], x[3]);
+                        ptx::ld_shared_v4(abuf + cp, x[0], x[1], x[2], x[3]);
                         uint32_t w[4];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
@@ -664,7 +673,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                             const ptx::f2 x2 = ptx::make_f2_bits(x[k] << 16, x[k] & 0xffff0000u);
                             w[k] = pack_f2_bf16x2(mul_gelu_bwd2(a2, x2));
                         }
-                        ptx::st_shared_v4(pos, w[0], w[1], w[2], w[3]);
+                        ptx::st_shared_v4(buf + cp, w[0], w[1], w[2], w[3]);
                     }
                 } else {  // kEpiF32: 32 fp32 columns per step, 16 per thread
                     uint32_t r[16];
@@ -716,11 +725,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         }
                     }
                     ptx::bulk_commit_group();
-                    if (EPI == kEpiMulGeluGrad) {
-                        // slot of step gstep+AUX_AHEAD was stored SLOTS-AUX_AHEAD groups ago
-                        ptx::bulk_wait_group_read<(SLOTS > AUX_AHEAD ? SLOTS - AUX_AHEAD : 0)>();
-                        issue_aux(gstep + AUX_AHEAD);
-                    }
+                    // every thread has read this step's pre-activation buffer (barrier above): refill it
+                    if (EPI == kEpiMulGeluGrad) issue_aux(gstep + AUX_AHEAD);
                     if (SLOTS == 1) ptx::bulk_wait_group_read<0>();
                 }
                 __syncwarp();  // the single-lane block above rejoins its warp before collective ops

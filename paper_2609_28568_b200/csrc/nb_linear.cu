@@ -278,14 +278,14 @@ using FwdStore1 = GemmCfg<1, 256, 4, 2, false, false, kEpiStore>;
 using FwdGelu1 = GemmCfg<1, 256, 3, 4, false, false, kEpiGelu>;
 using FwdSwiglu1 = GemmCfg<1, 256, 3, 3, false, false, kEpiSwiglu>;
 using DgradStore1 = GemmCfg<1, 256, 4, 2, false, true, kEpiStore>;
-using DgradMulGelu1 = GemmCfg<1, 256, 3, 4, false, true, kEpiMulGeluGrad>;
+using DgradMulGelu1 = GemmCfg<1, 256, 2, 2, false, true, kEpiMulGeluGrad>;
 using WgradF32_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32>;
 using WgradBf16_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiStore>;
 using FwdStore2 = GemmCfg<2, 256, 6, 2, false, false, kEpiStore>;
 using FwdGelu2 = GemmCfg<2, 256, 5, 4, false, false, kEpiGelu>;
 using FwdSwiglu2 = GemmCfg<2, 256, 5, 3, false, false, kEpiSwiglu>;
 using DgradStore2 = GemmCfg<2, 256, 6, 2, false, true, kEpiStore>;
-using DgradMulGelu2 = GemmCfg<2, 256, 5, 4, false, true, kEpiMulGeluGrad>;
+using DgradMulGelu2 = GemmCfg<2, 256, 4, 2, false, true, kEpiMulGeluGrad>;
 using WgradF32_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32>;
 using WgradF32Bias1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32, true>;
 using WgradF32Bias2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32, true>;
@@ -306,6 +306,29 @@ template <class C1, class C2>
 int launch_gemm_auto(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
 {
     return use_pairs(a.M) ? launch_gemm<C2>(s, a, stream) : launch_gemm<C1>(s, a, stream);
+}
+
+// Split-K factor for wgrad: the one whose waves of (tiles x splits) units over `slots` resident
+// tiles take the least time, counting a fixed cost per unit (epilogue and pipeline ramp, about six
+// k-blocks' worth). Every (m, n, k-range) is covered exactly once whatever the choice.
+int choose_splits(int tiles, int kblocks, int slots)
+{
+    const int kUnitOverhead = 6;
+    int best = 1;
+    long long best_cost = -1;
+    const int max_splits = kblocks / 4 > 1 ? kblocks / 4 : 1;
+    for (int sp = 1; sp <= max_splits && sp <= 128; ++sp) {
+        const int kps = (kblocks + sp - 1) / sp;
+        const int eff = (kblocks + kps - 1) / kps;  // splits that are not empty
+        const long long units = 1ll * tiles * eff;
+        const long long waves = (units + slots - 1) / slots;
+        const long long cost = waves * (kps + kUnitOverhead);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = eff;
+        }
+    }
+    return best;
 }
 
 int ensure_workspace(DeviceState &s, size_t bytes)
@@ -518,9 +541,7 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
             const int tiles = ((a.M + tile_m - 1) / tile_m) * ((a.N + 255) / 256);
             const int kblocks = (a.K + kBlockK - 1) / kBlockK;
             const int slots = s->num_sms / (use_pairs(a.M) ? 2 : 1);  // tiles resident at once
-            int splits = (2 * slots + tiles - 1) / tiles;
-            if (splits > kblocks / 4) splits = kblocks / 4;
-            if (splits < 1) splits = 1;
+            const int splits = choose_splits(tiles, kblocks, slots);
             a.splits = splits;
             a.reduce = (accumulate || splits > 1) ? 1 : 0;
             if (!accumulate && splits > 1)
@@ -614,6 +635,24 @@ int nb_check_status(void)
 }
 
 int64_t nb_kernel_launches(void) { return g_launches.load(); }
+
+int nb_debug_split_plan(int64_t M, int64_t N, int64_t K, int slots, int tile_m, int *out)
+{
+    if (!out || M <= 0 || N <= 0 || K <= 0 || slots <= 0 || (tile_m != 128 && tile_m != 256))
+        return fail(NB_ERR_INVALID_ARG, "bad argument");
+    const int tiles_m = static_cast<int>((M + tile_m - 1) / tile_m);
+    const int tiles_n = static_cast<int>((N + 255) / 256);
+    const int kblocks = static_cast<int>((K + kBlockK - 1) / kBlockK);
+    int splits = choose_splits(tiles_m * tiles_n, kblocks, slots);
+    const int kps = (kblocks + splits - 1) / splits;  // as launch_gemm derives it
+    splits = (kblocks + kps - 1) / kps;
+    out[0] = tiles_m;
+    out[1] = tiles_n;
+    out[2] = splits;
+    out[3] = kps;
+    out[4] = kblocks;
+    return NB_OK;
+}
 
 int nb_debug_wait_timeout(int64_t limit_us)
 {

@@ -1,0 +1,73 @@
+"""Time one kind of library call on one shape (also the small case used for ncu captures).
+
+    python -m paper_2609_28568_b200.microbench KIND BT C OC [REPS]
+
+KIND: fwd, fwd_nobias, fwd_gelu, fwd_swiglu, dgrad, dgrad_fused (dgrad with the producer's GELU
+backward in the epilogue), wgrad (accumulating), wgrad_bias (wgrad with the fused bias gradient),
+dbias (stand-alone column reduction), bwd (dgrad + wgrad + dbias in one call).
+Prints microseconds per call and TFLOP/s from CUDA events around REPS back-to-back calls.
+"""
+from __future__ import annotations
+
+import sys
+
+import torch
+
+from . import binding as nb
+from . import synth
+
+
+def main(argv) -> int:
+    if len(argv) < 5:
+        print(__doc__)
+        return 2
+    kind, BT, C, OC = argv[1], int(argv[2]), int(argv[3]), int(argv[4])
+    reps = int(argv[5]) if len(argv) > 5 else 20
+    dev = "cuda"
+    bf, f32 = torch.bfloat16, torch.float32
+    inp = synth.normal(1, (BT, C), 1.0, dev)
+    w = synth.normal(2, (OC, C), 0.02, dev)
+    b = synth.normal(3, (OC,), 0.02, dev)
+    dout = synth.normal(4, (BT, OC), 1e-3, dev)
+    ipre = synth.normal(5, (BT, C), 1.0, dev)
+    out = torch.empty((BT, OC), dtype=bf, device=dev)
+    pre = torch.empty((BT, OC), dtype=bf, device=dev)
+    dinp = torch.empty((BT, C), dtype=bf, device=dev)
+    dw = torch.zeros((OC, C), dtype=f32, device=dev)
+    db = torch.zeros((OC,), dtype=f32, device=dev)
+    calls = {
+        "fwd": lambda: nb.nb_linear_forward_ex(out, None, inp, w, b, BT, C, OC, nb.ACT_NONE),
+        "fwd_nobias": lambda: nb.nb_linear_forward_ex(out, None, inp, w, None, BT, C, OC, nb.ACT_NONE),
+        "fwd_gelu": lambda: nb.nb_linear_forward_ex(out, pre, inp, w, b, BT, C, OC, nb.ACT_GELU),
+        "fwd_swiglu": lambda: nb.nb_linear_forward_ex(out, pre, inp, w, None, BT, C, OC, nb.ACT_SWIGLU),
+        "dgrad": lambda: nb.nb_linear_backward_ex(dinp, None, None, dout, None, w, None, None, BT, C, OC, 0, 0),
+        "dgrad_fused": lambda: nb.nb_linear_backward_ex(dinp, None, None, dout, None, w, None, ipre, BT, C,
+                                                        OC, 0, 0),
+        "wgrad": lambda: nb.nb_linear_backward_ex(None, dw, None, dout, inp, None, None, None, BT, C, OC, 0, 1),
+        "wgrad_bias": lambda: nb.nb_linear_backward_ex(None, dw, db, dout, inp, None, None, None, BT, C, OC,
+                                                       0, 1),
+        "dbias": lambda: nb.nb_reduce_dbias(db, dout, BT, OC, 1),
+        "bwd": lambda: nb.nb_linear_backward_ex(dinp, dw, db, dout, inp, w, None, None, BT, C, OC, 0, 1),
+    }
+    if kind not in calls:
+        print(__doc__)
+        return 2
+    call = calls[kind]
+    for _ in range(2):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    nb.nb_check_status()
+    ms = e0.elapsed_time(e1) / reps
+    flops = 2 * BT * C * OC * (2 if kind == "bwd" else 1)
+    print(f"{kind} BT={BT} C={C} OC={OC}: {ms * 1e3:.1f} us/call  {flops / ms / 1e9:.1f} TFLOP/s")
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main(sys.argv))

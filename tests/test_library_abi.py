@@ -78,3 +78,25 @@ def test_binding_has_no_cpu_path(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(RuntimeError, match="missing"):
         binding.lib()
+
+
+def test_wgrad_split_plan_covers_every_k_block_once(L):
+    """Host logic: whatever split-K factor is chosen, the units partition (tile, k-block) space."""
+    shapes_ = [(2304, 768, 16384), (768, 768, 16384), (3072, 768, 16384), (768, 3072, 16384),
+               (50304, 768, 16384), (1024, 1024, 16384), (6144, 1024, 16384), (200, 72, 136),
+               (3072, 768, 128), (8, 8, 1), (776, 328, 5000)]
+    for M, N, K in shapes_:
+        for slots, tile_m in ((148, 128), (74, 256)):
+            tm, tn, splits, kps, kblocks = binding.nb_debug_split_plan(M, N, K, slots, tile_m)
+            assert tm == -(-M // tile_m) and tn == -(-N // 256) and kblocks == -(-K // 64)
+            assert 1 <= splits <= kblocks and kps >= 1
+            covered = [0] * kblocks
+            for s in range(splits):
+                lo, hi = s * kps, min((s + 1) * kps, kblocks)
+                assert lo < hi, "empty split"
+                for kb in range(lo, hi):
+                    covered[kb] += 1
+            assert covered == [1] * kblocks
+            # the chosen factor never leaves more than a wave's worth of imbalance on big problems
+            if kblocks >= 64 and tm * tn <= slots:
+                assert tm * tn * splits >= slots // 2

@@ -169,6 +169,16 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """The slowest rank's figure (a job is as slow as its slowest replica)."""
+    if dist is None:
+        return value
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 # ------------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -255,11 +265,7 @@ def main():
     barrier()
     launches = nb.nb_kernel_launches() - launches0
     nb.nb_check_status()
-    elapsed_ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     ms_per_step = elapsed_ms / args.steps
     tflops = world * flops_step / (ms_per_step * 1e-3) / 1e12
     tokens_per_s = world * tokens_step / (ms_per_step * 1e-3)
@@ -397,11 +403,7 @@ def measure_e2e(torch, nb, stack, args, dist, dev, flops_step, world):
     ev1.record()
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3
-    ms = max(ev0.elapsed_time(ev1), wall_ms) / args.e2e_steps
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(max(ev0.elapsed_time(ev1), wall_ms) / args.e2e_steps, dist, dev)
     nb.nb_check_status()
     return {"value": world * flops_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ms,

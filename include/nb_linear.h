@@ -113,9 +113,11 @@ int nb_linear_forward_ex(void *out, void *pre_act, const void *inp, const void *
  * BT == 0: dinp untouched, dweight/dbias zeroed when accumulate == 0.
  *
  * When pre_act != NULL, dz is first written to the library's device workspace
- * (BT*OC bf16, allocated on first need with cudaMalloc and kept). Summation order of
- * dweight/dbias across row blocks is not fixed, so results may differ in the last
- * bits between runs.
+ * (BT*OC bf16, allocated on first need with cudaMalloc and kept). When both dweight
+ * and dbias are requested, the bias gradient is summed inside the wgrad kernel from the
+ * dz tiles it already holds in shared memory. Summation order of dweight/dbias across
+ * row blocks is not fixed (split-K reduce-adds, atomics), so results may differ in the
+ * last bits between runs.
  */
 int nb_linear_backward(void *dinp, void *dweight, void *dbias, const void *dout,
                        const void *inp, const void *weight, const void *pre_act, int64_t BT,

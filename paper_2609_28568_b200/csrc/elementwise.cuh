@@ -94,19 +94,31 @@ dbias_kernel(float *__restrict__ dbias, const __nv_bfloat16 *__restrict__ dz, lo
         for (int k = 0; k < 8; ++k) acc[h][k] = 0.0f;
     const bool in0 = col0 + cv * 8 < OC;
     const bool in1 = col0 + 64 + cv * 8 < OC;
-    for (long long r = r_begin + warp * 4 + rs; r < r_end; r += 32) {
-        const __nv_bfloat16 *rowp = dz + r * OC + col0 + cv * 8;
-        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = make_uint4(0, 0, 0, 0);
-        if (in0) v0 = __ldg(reinterpret_cast<const uint4 *>(rowp));
-        if (in1) v1 = __ldg(reinterpret_cast<const uint4 *>(rowp + 64));
-        const uint32_t a[4] = {v0.x, v0.y, v0.z, v0.w};
-        const uint32_t b[4] = {v1.x, v1.y, v1.z, v1.w};
+    // four rows per thread in flight (eight 128-bit loads) to cover the DRAM latency
+    for (long long r0 = r_begin + warp * 4 + rs; r0 < r_end; r0 += 128) {
+        uint4 v0[4], v1[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            acc[0][2 * k] += ptx::bf16_lo(a[k]);
-            acc[0][2 * k + 1] += ptx::bf16_hi(a[k]);
-            acc[1][2 * k] += ptx::bf16_lo(b[k]);
-            acc[1][2 * k + 1] += ptx::bf16_hi(b[k]);
+        for (int i = 0; i < 4; ++i) {
+            const long long r = r0 + 32 * i;
+            v0[i] = make_uint4(0, 0, 0, 0);
+            v1[i] = make_uint4(0, 0, 0, 0);
+            if (r < r_end) {
+                const __nv_bfloat16 *rowp = dz + r * OC + col0 + cv * 8;
+                if (in0) v0[i] = __ldg(reinterpret_cast<const uint4 *>(rowp));
+                if (in1) v1[i] = __ldg(reinterpret_cast<const uint4 *>(rowp + 64));
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t a[4] = {v0[i].x, v0[i].y, v0[i].z, v0[i].w};
+            const uint32_t b[4] = {v1[i].x, v1[i].y, v1[i].z, v1[i].w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[0][2 * k] += ptx::bf16_lo(a[k]);
+                acc[0][2 * k + 1] += ptx::bf16_hi(a[k]);
+                acc[1][2 * k] += ptx::bf16_lo(b[k]);
+                acc[1][2 * k + 1] += ptx::bf16_hi(b[k]);
+            }
         }
     }
     __syncthreads();

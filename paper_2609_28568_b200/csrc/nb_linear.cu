@@ -352,10 +352,10 @@ int launch_dbias(DeviceState &s, float *dbias, const void *dz, int64_t BT, int64
     if (!accumulate) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
     if (BT == 0) return NB_OK;
     const int col_blocks = static_cast<int>((OC + kDbiasCols - 1) / kDbiasCols);
-    long long want_row_blocks = (8ll * s.num_sms + col_blocks - 1) / col_blocks;
+    long long want_row_blocks = (6ll * s.num_sms + col_blocks - 1) / col_blocks;
     long long rows_per_block = (BT + want_row_blocks - 1) / want_row_blocks;
-    rows_per_block = ((rows_per_block + 31) / 32) * 32;
-    if (rows_per_block < 32) rows_per_block = 32;
+    rows_per_block = ((rows_per_block + 127) / 128) * 128;  // a block sweeps 128 rows per iteration
+    if (rows_per_block < 128) rows_per_block = 128;
     const long long row_blocks = (BT + rows_per_block - 1) / rows_per_block;
     if (row_blocks > 65535) return fail(NB_ERR_UNSUPPORTED, "BT too large for the dbias grid");
     dim3 grid(col_blocks, static_cast<unsigned>(row_blocks));

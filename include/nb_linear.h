@@ -153,6 +153,15 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
 int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int accumulate);
 
 /*
+ * Master-weight cast: dst[i] = bf16(src[i]), round to nearest even, for n elements.
+ * (paper: Method/Optimisation and precision keeps fp32 master weights and bf16 compute copies;
+ * Results/Speed, the table of levers: the cast is done once per optimizer step and reused by
+ * every micro-step.) src fp32 and dst bf16 are device pointers, 16-byte aligned; n >= 0.
+ * Infinities are kept, values beyond the largest finite bf16 round to infinity, NaN stays NaN.
+ */
+int nb_cast_f32_to_bf16(void *dst, const void *src, int64_t n, void *stream);
+
+/*
  * Bias gradient of a GELU layer without any allocation (the paper has no counterpart; this
  * exists for callers that must not allocate device memory):
  *

@@ -176,3 +176,13 @@ def reduce_dbias(dout, dbias=None, accumulate: bool = False):
     if rc != 0:
         raise ValueError("oracle reduce_dbias rejected the request")
     return dbias
+
+
+def cast_f32_bf16(src):
+    """fp32 -> bf16 bit patterns (uint16), round to nearest even."""
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    dst = np.empty(src.shape, dtype=np.uint16)
+    fn = _load().nbo_cast_f32_bf16
+    fn.restype = None
+    fn(_p(dst), _p(src), ctypes.c_int64(src.size))
+    return dst

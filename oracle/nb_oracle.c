@@ -57,6 +57,30 @@ int nbo_reduce_dbias_f64(double *dbias, const float *dout, int64_t BT, int64_t O
     return 0;
 }
 
+/*
+ * fp32 -> bf16, round to nearest, ties to even (the master-weight cast done once per optimizer
+ * step; paper: Results/Speed, the table of levers, "master-cast reuse across micro-steps").
+ * Written on the bit patterns: keep the top 16 bits, add one when the discarded half is above
+ * one half of the last kept bit, or exactly one half and the kept value is odd. Infinities stay,
+ * a carry out of the largest finite value gives infinity, NaN stays NaN (quiet, sign kept).
+ */
+void nbo_cast_f32_bf16(uint16_t *dst, const float *src, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        uint32_t u;
+        memcpy(&u, &src[i], 4);
+        const uint32_t exp = (u >> 23) & 0xFFu, man = u & 0x7FFFFFu;
+        if (exp == 0xFFu && man != 0) { /* NaN */
+            dst[i] = (uint16_t)((u >> 16) | 0x0040u);
+            continue;
+        }
+        const uint32_t kept = u >> 16, rest = u & 0xFFFFu;
+        uint32_t r = kept;
+        if (rest > 0x8000u || (rest == 0x8000u && (kept & 1u))) r = kept + 1u;
+        dst[i] = (uint16_t)r;
+    }
+}
+
 int nbo_num_threads(void)
 {
 #ifdef _OPENMP

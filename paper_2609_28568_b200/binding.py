@@ -23,7 +23,7 @@ EXPORTS = (
     "nb_linear_forward", "nb_linear_forward_ex", "nb_linear_backward", "nb_linear_backward_ex",
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
     "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
-    "nb_debug_split_plan",
+    "nb_debug_split_plan", "nb_cast_f32_to_bf16",
 )
 
 _lib = None
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.nb_debug_wait_timeout.argtypes = [_i64]
         L.nb_kernel_launches.restype = _i64
         L.nb_gelu_dbias_noalloc.argtypes = [_vp, _vp, _vp, _i64, _i64, _int, _vp]
+        L.nb_cast_f32_to_bf16.argtypes = [_vp, _vp, _i64, _vp]
         L.nb_debug_split_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int)]
         _lib = L
     return _lib
@@ -150,6 +151,11 @@ def nb_gelu_dbias_noalloc(dbias, dout, pre_act, BT, OC, accumulate, stream=None)
     the library: for callers that may not allocate device memory. BT*OC <= NOALLOC_MAX_ELEMS."""
     _check(lib().nb_gelu_dbias_noalloc(_ptr(dbias), _ptr(dout), _ptr(pre_act), BT, OC,
                                        int(accumulate), _stream() if stream is None else stream))
+
+
+def nb_cast_f32_to_bf16(dst, src, n, stream=None) -> None:
+    """Master-weight cast: dst (bf16) = src (fp32), round to nearest even."""
+    _check(lib().nb_cast_f32_to_bf16(_ptr(dst), _ptr(src), n, _stream() if stream is None else stream))
 
 
 def nb_debug_split_plan(M: int, N: int, K: int, slots: int, tile_m: int):

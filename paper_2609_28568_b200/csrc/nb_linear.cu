@@ -592,6 +592,24 @@ int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int a
     return launch_dbias(*s, static_cast<float *>(dbias), dout, BT, OC, accumulate, g_stream);
 }
 
+int nb_cast_f32_to_bf16(void *dst, const void *src, int64_t n, void *stream_)
+{
+    if (n < 0) return fail(NB_ERR_INVALID_ARG, "negative size");
+    if (n == 0) return NB_OK;
+    if (!dst || !src) return fail(NB_ERR_INVALID_ARG, "dst and src must not be NULL");
+    if (!aligned16(dst) || !aligned16(src))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    cast_f32_bf16_kernel<<<elementwise_grid(*s, n / 8 + 1), 256, 0, static_cast<cudaStream_t>(stream_)>>>(
+        static_cast<__nv_bfloat16 *>(dst), static_cast<const float *>(src), n);
+    NB_CUDA(cudaGetLastError());
+    ++g_launches;
+    return NB_OK;
+}
+
 int nb_workspace_reserve(int64_t bytes)
 {
     if (bytes < 0) return fail(NB_ERR_INVALID_ARG, "negative size");

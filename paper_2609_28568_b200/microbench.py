@@ -4,7 +4,8 @@
 
 KIND: fwd, fwd_nobias, fwd_gelu, fwd_swiglu, dgrad, dgrad_fused (dgrad with the producer's GELU
 backward in the epilogue), wgrad (accumulating), wgrad_bias (wgrad with the fused bias gradient),
-dbias (stand-alone column reduction), bwd (dgrad + wgrad + dbias in one call).
+dbias (stand-alone column reduction), bwd (dgrad + wgrad + dbias in one call), cast (fp32 -> bf16
+master-weight cast of OC*C elements; reports GB/s as "TFLOP/s"-free line).
 Prints microseconds per call and TFLOP/s from CUDA events around REPS back-to-back calls.
 """
 from __future__ import annotations
@@ -49,6 +50,11 @@ def main(argv) -> int:
         "dbias": lambda: nb.nb_reduce_dbias(db, dout, BT, OC, 1),
         "bwd": lambda: nb.nb_linear_backward_ex(dinp, dw, db, dout, inp, w, None, None, BT, C, OC, 0, 1),
     }
+    if kind == "cast":
+        n = OC * C
+        src = torch.randn(n, dtype=f32, device=dev)
+        dst = torch.empty(n, dtype=bf, device=dev)
+        calls["cast"] = lambda: nb.nb_cast_f32_to_bf16(dst, src, n)
     if kind not in calls:
         print(__doc__)
         return 2
@@ -64,6 +70,9 @@ def main(argv) -> int:
     torch.cuda.synchronize()
     nb.nb_check_status()
     ms = e0.elapsed_time(e1) / reps
+    if kind == "cast":
+        print(f"cast n={OC * C}: {ms * 1e3:.1f} us/call  {OC * C * 6 / ms / 1e6:.1f} GB/s")
+        return 0
     flops = 2 * BT * C * OC * (2 if kind == "bwd" else 1)
     print(f"{kind} BT={BT} C={C} OC={OC}: {ms * 1e3:.1f} us/call  {flops / ms / 1e9:.1f} TFLOP/s")
     return 0

@@ -439,3 +439,23 @@ def test_run_to_run_determinism_report():
     print("determinism: forward bitwise, dgrad bitwise, dweight bitwise =",
           all(torch.equal(dws[i], dws[0]) for i in (1, 2)), ", dbias bitwise =",
           all(torch.equal(dbs[i], dbs[0]) for i in (1, 2)))
+
+
+def test_master_weight_cast_bit_exact():
+    """fp32 -> bf16 cast: integer work, so bit-exact against the oracle, ragged tails included."""
+    g = torch.Generator().manual_seed(9)
+    for n in (1, 7, 8, 9, 4099, 768 * 2304, 50304 * 768 + 5):
+        x = (torch.randn(n, generator=g) * 0.02)
+        if n > 64:  # special values: ties, carries, infinities, subnormals, zeros
+            sp = torch.tensor([0x3F808000, 0x3F818000, 0x3F808001, 0x7F7FFFFF, 0x7F800000, 0x00008000,
+                               0x00018000, 0x00000000], dtype=torch.int64).to(torch.int32).view(torch.float32)
+            x[:8] = sp
+            x[8:16] = -sp
+        xd = x.to(DEV)
+        dst = Guarded((n,), torch.bfloat16) if n % 8 == 0 else None
+        out = dst.t if dst else torch.empty(n, dtype=torch.bfloat16, device=DEV)
+        nb.nb_cast_f32_to_bf16(out, xd, n)
+        got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got, oracle.cast_f32_bf16(x.numpy())), n
+        if dst:
+            dst.check("cast")

@@ -341,3 +341,38 @@ def test_malformed_requests_are_rejected():
 def test_threads_reported():
     assert oracle.num_threads() >= 1
     assert math.isfinite(oracle.num_threads())
+
+
+# ---------------------------------------------------------------- fp32 -> bf16 cast
+
+def test_cast_against_library_and_hand_cases():
+    """The bit-level cast equals the library's conversion, and the tie / carry / special cases hold."""
+    g = torch.Generator().manual_seed(5)
+    x = torch.randn(200000, generator=g) * torch.exp(torch.randn(200000, generator=g) * 8)
+    bits = x.view(torch.int32).clone()
+    bits[:1000] = torch.randint(-2**31, 2**31 - 1, (1000,), generator=g, dtype=torch.int64).to(torch.int32)
+    x = bits.view(torch.float32)
+    got = oracle.cast_f32_bf16(x.numpy())
+    want = x.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    nan = np.isnan(x.numpy())
+    assert np.array_equal(got[~nan], want[~nan])
+    assert np.all((got[nan] & 0x7F80) == 0x7F80) and np.all((got[nan] & 0x007F) != 0)  # still NaN
+
+    def f(bits32):
+        return np.array([bits32], dtype=np.uint32).view(np.float32)
+
+    cases = [
+        (0x3F800000, 0x3F80),  # 1.0
+        (0x3F808000, 0x3F80),  # 1 + 2^-8: a tie, kept value even -> stays
+        (0x3F818000, 0x3F82),  # 1 + 3*2^-8: a tie, kept value odd -> up
+        (0x3F808001, 0x3F81),  # just above the tie -> up
+        (0x3F807FFF, 0x3F80),  # just below the tie -> down
+        (0x7F7FFFFF, 0x7F80),  # largest fp32 rounds to +inf
+        (0x7F800000, 0x7F80), (0xFF800000, 0xFF80),  # infinities
+        (0x00000000, 0x0000), (0x80000000, 0x8000),  # signed zeros
+        (0x00008000, 0x0000),  # subnormal tie to even (zero)
+        (0x00018000, 0x0002),  # subnormal tie, odd -> up
+        (0xBF808001, 0xBF81),  # negative, above the tie in magnitude
+    ]
+    for b32, b16 in cases:
+        assert oracle.cast_f32_bf16(f(b32))[0] == b16, hex(b32)

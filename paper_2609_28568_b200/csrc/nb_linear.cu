@@ -239,7 +239,10 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     if (splits > p.kblocks) splits = p.kblocks;
     p.kblocks_per_split = (p.kblocks + splits - 1) / splits;
     p.splits = (p.kblocks + p.kblocks_per_split - 1) / p.kblocks_per_split;
-    p.group_m = 16 / Cfg::CG;
+    // rasterisation: units walk `group_m` row tiles for each column tile before moving to the next
+    // column tile. Many column tiles (the head): a tall group keeps the weight tiles' reuse in L2;
+    // few column tiles: a short group keeps the row tiles' (measured on B200, 1-2 % either way)
+    p.group_m = (p.tiles_n >= 64 ? 64 : p.tiles_n <= 4 ? 4 : 16) / Cfg::CG;
     p.swiglu_h = a.swiglu_h;
     p.reduce = a.reduce;
     p.bias = static_cast<const __nv_bfloat16 *>(a.bias);

@@ -318,7 +318,7 @@ def main():
         gemm_ms += ms
     peaks, peak_src = load_peaks()
     # the GPU is under load for warm-up + timed + breakdown steps back to back: over a second of
-    # that is the "kernel timed inside a long step" case, judged against the sustained peak
+    # that is the "kernel timed inside a long step" case, compared with the sustained peak
     long_step = ms_per_step * (args.warmup + 2 * args.steps) > 1000.0
     peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
     achieved_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0

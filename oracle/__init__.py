@@ -186,3 +186,23 @@ def cast_f32_bf16(src):
     fn.restype = None
     fn(_p(dst), _p(src), ctypes.c_int64(src.size))
     return dst
+
+
+def cross_entropy(logits, targets, V: int, gscale: float = 1.0, want_grad: bool = True):
+    """Per-row ``(loss, lse, dlogits)`` of the cross-entropy over the first V columns of ``logits``.
+
+    ``dlogits = gscale * (softmax - onehot)`` on the first V columns and 0 on the padding ones.
+    """
+    logits = _f32c(logits)
+    BT, Vp = logits.shape
+    targets = np.ascontiguousarray(targets, dtype=np.int32)
+    loss = np.empty((BT,), dtype=np.float64)
+    lse = np.empty((BT,), dtype=np.float64)
+    dl = np.empty((BT, Vp), dtype=np.float64) if want_grad else None
+    fn = _load().nbo_cross_entropy_f64
+    fn.restype = ctypes.c_int
+    rc = fn(_p(loss), _p(lse), _p(dl), _p(logits), _p(targets), ctypes.c_int64(BT), ctypes.c_int64(Vp),
+            ctypes.c_int64(V), ctypes.c_double(gscale))
+    if rc != 0:
+        raise ValueError("oracle cross_entropy rejected the request")
+    return loss, lse, dl

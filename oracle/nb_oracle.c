@@ -81,6 +81,42 @@ void nbo_cast_f32_bf16(uint16_t *dst, const float *src, int64_t n)
     }
 }
 
+/*
+ * Cross-entropy of the head's logits over the first V of Vp columns (paper: Figure 1, "cross-entropy
+ * over the first 50,257; padding rows get no probability and no gradient"; loss in f32).
+ *   lse[i]       = log sum_{j<V} exp(logits[i,j])
+ *   loss[i]      = lse[i] - logits[i, target[i]]
+ *   dlogits[i,j] = gscale * (exp(logits[i,j] - lse[i]) - [j == target[i]])   for j <  V
+ *                = 0                                                          for j >= V
+ * logits are floats holding the stored bf16 values; everything else is double. dlogits may be
+ * NULL. Returns -1 on a malformed request (a target outside [0, V) included).
+ */
+int nbo_cross_entropy_f64(double *loss, double *lse, double *dlogits, const float *logits,
+                          const int32_t *targets, int64_t BT, int64_t Vp, int64_t V, double gscale)
+{
+    if (!loss || !lse || !logits || !targets || BT < 0 || V <= 0 || Vp < V) return -1;
+    for (int64_t i = 0; i < BT; ++i)
+        if (targets[i] < 0 || targets[i] >= V) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < BT; ++i) {
+        const float *row = logits + i * Vp;
+        double mx = (double)row[0];
+        for (int64_t j = 1; j < V; ++j)
+            if ((double)row[j] > mx) mx = (double)row[j];
+        double sum = 0.0;
+        for (int64_t j = 0; j < V; ++j) sum += exp((double)row[j] - mx);
+        lse[i] = mx + log(sum);
+        loss[i] = lse[i] - (double)row[targets[i]];
+        if (dlogits) {
+            double *d = dlogits + i * Vp;
+            for (int64_t j = 0; j < V; ++j)
+                d[j] = gscale * (exp((double)row[j] - lse[i]) - (j == targets[i] ? 1.0 : 0.0));
+            for (int64_t j = V; j < Vp; ++j) d[j] = 0.0;
+        }
+    }
+    return 0;
+}
+
 int nbo_num_threads(void)
 {
 #ifdef _OPENMP

@@ -376,3 +376,45 @@ def test_cast_against_library_and_hand_cases():
     ]
     for b32, b16 in cases:
         assert oracle.cast_f32_bf16(f(b32))[0] == b16, hex(b32)
+
+
+# ---------------------------------------------------------------- cross-entropy over the real vocabulary
+
+def test_cross_entropy_against_library_autograd():
+    BT, Vp, V = 23, 48, 41
+    g = torch.Generator().manual_seed(12)
+    logits = (torch.randn(BT, Vp, generator=g) * 3).to(torch.bfloat16).float()
+    targets = torch.randint(0, V, (BT,), generator=g)
+    gscale = 1.0 / BT
+    x = logits.double().requires_grad_(True)
+    per_row = F.cross_entropy(x[:, :V], targets, reduction="none")
+    (gx,) = torch.autograd.grad((per_row * gscale).sum(), x)
+    loss, lse, dl = oracle.cross_entropy(logits.numpy(), targets.numpy(), V, gscale)
+    assert np.max(np.abs(loss - per_row.detach().numpy())) < 1e-12
+    assert np.max(np.abs(lse - torch.logsumexp(x[:, :V], 1).detach().numpy())) < 1e-12
+    assert np.max(np.abs(dl - gx.numpy())) < 1e-15
+    assert np.all(dl[:, V:] == 0.0)                      # padding columns: no gradient
+    assert np.max(np.abs(dl.sum(1))) < 1e-15             # softmax - onehot sums to zero per row
+
+
+def test_cross_entropy_closed_forms():
+    BT, Vp, V = 5, 16, 11
+    # equal logits: uniform distribution over the V real columns, whatever the padding holds
+    logits = np.full((BT, Vp), 0.75, dtype=np.float32)
+    logits[:, V:] = 100.0
+    t = np.arange(BT) % V
+    loss, lse, dl = oracle.cross_entropy(logits, t, V)
+    assert np.allclose(loss, math.log(V), atol=1e-14) and np.allclose(lse, 0.75 + math.log(V), atol=1e-14)
+    assert np.allclose(dl[0, 1:V], 1.0 / V, atol=1e-15) and abs(dl[0, 0] - (1.0 / V - 1.0)) < 1e-15
+    # one dominant logit on the target: loss -> 0, gradient -> 0
+    logits = np.zeros((1, Vp), dtype=np.float32)
+    logits[0, 3] = 80.0
+    loss, _, dl = oracle.cross_entropy(logits, [3], V)
+    assert loss[0] < 1e-30 + 1e-12 and np.max(np.abs(dl)) < 1e-12
+    # shift invariance of the loss, and rejection of an out-of-range target
+    a = np.random.default_rng(0).standard_normal((4, Vp)).astype(np.float32)
+    l1, _, _ = oracle.cross_entropy(a, [0, 1, 2, 3], V, want_grad=False)
+    l2, _, _ = oracle.cross_entropy(a + np.float32(2.0), [0, 1, 2, 3], V, want_grad=False)
+    assert np.max(np.abs(l1 - l2)) < 1e-6
+    with pytest.raises(ValueError):
+        oracle.cross_entropy(a, [0, 1, 2, V], V)

@@ -153,6 +153,31 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
 int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int accumulate);
 
 /*
+ * Head with fused cross-entropy statistics (paper: Figure 1, "cross-entropy over the first 50,257;
+ * padding rows get no probability and no gradient", loss in f32; Results/Speed lists the
+ * cross-entropy forward and backward as separate kernels next to the head's GEMMs).
+ *
+ * nb_lm_head_ce_forward: logits = inp . weight^T (bf16, [BT, Vp], stored as by nb_linear_forward),
+ * and, in the same pass, from the stored (rounded) logits of the first V columns:
+ *     lse[i]  = log sum_{j < V} exp(logits[i, j])          fp32 [BT]
+ *     loss[i] = lse[i] - logits[i, targets[i]]             fp32 [BT]
+ * The GEMM epilogue keeps per-row (max, sum of exp) per column tile; a small second kernel
+ * combines them, so the logits are never re-read for the softmax normaliser. targets: int32
+ * [BT] on the device, each in [0, V); an out-of-range target yields NaN in loss[i]. Vp and C
+ * multiples of 8, 0 < V <= Vp. Uses the library workspace (BT * 2*ceil(Vp/256) * 8 bytes).
+ *
+ * nb_ce_backward: dlogits[i, j] = gscale * (exp(logits[i, j] - lse[i]) - [j == targets[i]]) for
+ * j < V and 0 for j >= V, bf16 [BT, Vp]; dlogits may be the logits buffer itself (in place). Its
+ * result is the `dout` of nb_linear_backward for the head. gscale is the upstream gradient of
+ * every row's loss (1/BT for a mean over the micro-batch, times 1/accumulation steps).
+ */
+int nb_lm_head_ce_forward(void *logits, void *loss, void *lse, const void *inp, const void *weight,
+                          const void *targets, int64_t BT, int64_t C, int64_t Vp, int64_t V,
+                          void *stream);
+int nb_ce_backward(void *dlogits, const void *logits, const void *lse, const void *targets,
+                   float gscale, int64_t BT, int64_t Vp, int64_t V, void *stream);
+
+/*
  * Master-weight cast: dst[i] = bf16(src[i]), round to nearest even, for n elements.
  * (paper: Method/Optimisation and precision keeps fp32 master weights and bf16 compute copies;
  * Results/Speed, the table of levers: the cast is done once per optimizer step and reused by

@@ -23,7 +23,7 @@ EXPORTS = (
     "nb_linear_forward", "nb_linear_forward_ex", "nb_linear_backward", "nb_linear_backward_ex",
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
     "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
-    "nb_debug_split_plan", "nb_cast_f32_to_bf16",
+    "nb_debug_split_plan", "nb_cast_f32_to_bf16", "nb_lm_head_ce_forward", "nb_ce_backward",
 )
 
 _lib = None
@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.nb_kernel_launches.restype = _i64
         L.nb_gelu_dbias_noalloc.argtypes = [_vp, _vp, _vp, _i64, _i64, _int, _vp]
         L.nb_cast_f32_to_bf16.argtypes = [_vp, _vp, _i64, _vp]
+        L.nb_lm_head_ce_forward.argtypes = [_vp] * 6 + [_i64] * 4 + [_vp]
+        L.nb_ce_backward.argtypes = [_vp] * 4 + [ctypes.c_float] + [_i64] * 3 + [_vp]
         L.nb_debug_split_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int)]
         _lib = L
     return _lib
@@ -151,6 +153,19 @@ def nb_gelu_dbias_noalloc(dbias, dout, pre_act, BT, OC, accumulate, stream=None)
     the library: for callers that may not allocate device memory. BT*OC <= NOALLOC_MAX_ELEMS."""
     _check(lib().nb_gelu_dbias_noalloc(_ptr(dbias), _ptr(dout), _ptr(pre_act), BT, OC,
                                        int(accumulate), _stream() if stream is None else stream))
+
+
+def nb_lm_head_ce_forward(logits, loss, lse, inp, weight, targets, BT, C, Vp, V, stream=None) -> None:
+    """Head GEMM with the softmax statistics of the first V columns fused in: logits, loss, lse."""
+    _check(lib().nb_lm_head_ce_forward(_ptr(logits), _ptr(loss), _ptr(lse), _ptr(inp), _ptr(weight),
+                                       _ptr(targets), BT, C, Vp, V,
+                                       _stream() if stream is None else stream))
+
+
+def nb_ce_backward(dlogits, logits, lse, targets, gscale, BT, Vp, V, stream=None) -> None:
+    """dlogits = gscale * (softmax - onehot) on the first V columns, 0 on the padding."""
+    _check(lib().nb_ce_backward(_ptr(dlogits), _ptr(logits), _ptr(lse), _ptr(targets), gscale, BT, Vp, V,
+                                _stream() if stream is None else stream))
 
 
 def nb_cast_f32_to_bf16(dst, src, n, stream=None) -> None:

@@ -157,6 +157,67 @@ cast_f32_bf16_kernel(__nv_bfloat16 *__restrict__ dst, const float *__restrict__ 
     for (long long i = nvec * 8 + t0; i < n; i += stride) dst[i] = __float2bfloat16_rn(src[i]);
 }
 
+// Cross-entropy over the first V columns of the head's logits, from the per-tile softmax statistics
+// the forward GEMM wrote: one warp per row combines the partial (max, sum exp) pairs into
+// lse = log sum_j exp(logit_j) and loss = lse - logit[target]. A target outside [0, V) gives NaN.
+__global__ void __launch_bounds__(256)
+ce_reduce_kernel(float *__restrict__ loss, float *__restrict__ lse, const float2 *__restrict__ stats,
+                 int stats_ld, const __nv_bfloat16 *__restrict__ logits, long long ld,
+                 const int *__restrict__ targets, long long BT, int V)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = static_cast<long long>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+    if (row >= BT) return;
+    const float2 *st = stats + row * stats_ld;
+    float m = -INFINITY;
+    for (int k = lane; k < stats_ld; k += 32) m = fmaxf(m, st[k].x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float s = 0.0f;
+    for (int k = lane; k < stats_ld; k += 32) {
+        const float2 v = st[k];
+        if (v.x > -INFINITY) s += v.y * __expf(v.x - m);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+        const float l = m + __logf(s);
+        const int t = targets[row];
+        lse[row] = l;
+        loss[row] = (t >= 0 && t < V) ? l - __bfloat162float(logits[row * ld + t]) : NAN;
+    }
+}
+
+// dlogits = gscale * (softmax - onehot) on the first V columns, 0 on the padding columns;
+// 8 columns per thread (128-bit load and store). May run in place (dlogits == logits).
+__global__ void __launch_bounds__(256)
+ce_backward_kernel(uint4 *dlogits, const uint4 *logits, const float *__restrict__ lse,
+                   const int *__restrict__ targets, float gscale, long long BT, int vec_per_row, int V)
+{
+    const long long total = BT * vec_per_row;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += stride) {
+        const long long row = i / vec_per_row;
+        const int col0 = static_cast<int>(i - row * vec_per_row) * 8;
+        const uint4 v = logits[i];
+        const float l = lse[row] * 1.4426950408889634f;
+        const int t = targets[row];
+        const uint32_t x[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int c = col0 + 2 * k;
+            float p0 = ptx::ex2_approx(fmaf(ptx::bf16_lo(x[k]), 1.4426950408889634f, -l));
+            float p1 = ptx::ex2_approx(fmaf(ptx::bf16_hi(x[k]), 1.4426950408889634f, -l));
+            p0 = (c < V) ? gscale * (p0 - (c == t ? 1.0f : 0.0f)) : 0.0f;
+            p1 = (c + 1 < V) ? gscale * (p1 - (c + 1 == t ? 1.0f : 0.0f)) : 0.0f;
+            o[k] = ptx::pack_bf16x2(p0, p1);
+        }
+        dlogits[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 // Waits on a barrier that nothing signals, for at most limit_ns, then leaves normally.
 __global__ void wait_timeout_kernel(int *status, unsigned long long limit_ns)
 {

@@ -44,7 +44,9 @@ enum EpiMode : int {
     kEpiGelu = 1,         // E(bf16) = z = acc + bias ; D(bf16) = gelu(z)
     kEpiSwiglu = 2,       // E = z (gate | up planes) ; D[:, j] = silu(gate_j) * up_j
     kEpiMulGeluGrad = 3,  // D(bf16) = acc * gelu'(E)    (E is read)
-    kEpiF32 = 4           // D(fp32) = acc, stored or reduce-added
+    kEpiF32 = 4,          // D(fp32) = acc, stored or reduce-added
+    kEpiStoreStats = 5    // kEpiStore, plus per-row (max, sum of exp) of the stored values over the
+                          // tile's columns below v_real: the softmax statistics of the head's logits
 };
 
 struct GemmParams {
@@ -58,6 +60,9 @@ struct GemmParams {
     int reduce;             // kEpiF32: 1 reduce-add into D, 0 overwrite
     const __nv_bfloat16 *bias;  // [N] or nullptr
     float *dbias;               // wgrad with fused bias gradient: dbias[m] += sum_k A[m,k]
+    float2 *stats;              // kEpiStoreStats: [M, stats_ld] partial (max, sum exp) per row
+    int stats_ld;               //   two entries per column tile (one per column half of a step)
+    int v_real;                 //   columns >= v_real take no part in the statistics
     int *status;
     unsigned long long timeout_ns;
 };
@@ -326,7 +331,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // fall through to the common exit
     } else if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (every CTA)
-        if (lane == 0) {
+        // One elected lane; the election sits in a warp-uniform branch, the form in which the
+        // compiler hands coordinates to the TMA unit reliably (a thread-index test did not).
+        if (ptx::elect_one()) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -386,7 +393,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        if (rank == 0 && ptx::elect_one()) {
             constexpr uint32_t idesc = make_idesc(Cfg::TILE_M, BLOCK_N, Cfg::A_MN, Cfg::B_MN);
             int stage = 0;
             uint32_t phase = 0;
@@ -508,7 +515,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int q = warp & 3;
         const int hf = (warp - 2) >> 2;
         const int row = q * 32 + lane;
-        const bool leader = (threadIdx.x == 64);
+        // TMA stores and the bulk-group bookkeeping are issued by one elected lane of warp 2, always
+        // from a warp-uniform branch with the election at the point of use
+        const bool store_warp = (warp == 2);
         const int et = static_cast<int>(threadIdx.x) - 64;  // 0..255
         const uint32_t stg0 = smem + Cfg::OFF_STG;
         const uint32_t bias_s = smem + Cfg::OFF_BIAS;
@@ -535,11 +544,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t ab = aux_bar(static_cast<int>(slot));
             ptx::mbar_expect_tx(ab, kStgBytes);
             ptx::tma_load_2d(smem + Cfg::OFF_AUX + slot * kStgBytes, &tmE, ab, x,
-                             ptx::fresh(m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM));
+                             m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM);
         };
         if constexpr (EPI == kEpiMulGeluGrad) {
-            if (leader) {
-                for (int g = 0; g < AUX_AHEAD; ++g) issue_aux(static_cast<uint32_t>(g));
+            if (store_warp) {
+                if (ptx::elect_one()) {
+                    for (int g = 0; g < AUX_AHEAD; ++g) issue_aux(static_cast<uint32_t>(g));
+                }
             }
         }
         __syncwarp();
@@ -565,7 +576,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             decode_unit(p, u, m_blk, n_blk, split);
             const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
             const int n0 = (EPI == kEpiSwiglu) ? n_blk * 128 : n_blk * BLOCK_N;
-            if (EPI == kEpiStore || EPI == kEpiGelu || EPI == kEpiSwiglu) {
+            if (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiGelu || EPI == kEpiSwiglu) {
                 for (int i = et; i < BLOCK_N; i += kEpiThreads) {
                     int col;
                     if (EPI == kEpiSwiglu) col = (i < 128) ? (n0 + i) : (p.swiglu_h + n0 + i - 128);
@@ -585,17 +596,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                    static_cast<uint32_t>(acc * BLOCK_N);
 
+            float st_m = -INFINITY, st_s = 0.0f;  // kEpiStoreStats: this thread's row statistics
 #pragma unroll 1
             for (int c = 0; c < STEPS; ++c, ++gstep) {
                 const uint32_t slot = gstep % SLOTS;
                 const uint32_t buf = stg0 + slot * Cfg::BUFS_PER_STEP * kStgBytes;
 
-                if (EPI == kEpiStore || EPI == kEpiGelu) {
+                if (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiGelu) {
                     // this thread: columns [c*64 + hf*32, +32) of its row
                     const int col0 = c * 64 + hf * 32;
                     uint32_t r[32];
                     ptx::tmem_ld_32x32_wait(t_acc + col0, r);
                     if (c == STEPS - 1) release_acc(acc);  // accumulator fully read
+                    float sv[EPI == kEpiStoreStats ? 32 : 1];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         float4 b0, b1;
@@ -613,8 +626,38 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                             for (int k = 0; k < 4; ++k) z[k] = gelu_fwd2(z[k]);
                         }
-                        ptx::st_shared_v4(buf + pos, pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),
-                                          pack_f2_bf16x2(z[2]), pack_f2_bf16x2(z[3]));
+                        const uint32_t w0 = pack_f2_bf16x2(z[0]), w1 = pack_f2_bf16x2(z[1]),
+                                       w2 = pack_f2_bf16x2(z[2]), w3 = pack_f2_bf16x2(z[3]);
+                        ptx::st_shared_v4(buf + pos, w0, w1, w2, w3);
+                        if (EPI == kEpiStoreStats) {  // keep the eight stored (rounded) values
+                            sv[j * 8 + 0] = ptx::bf16_lo(w0); sv[j * 8 + 1] = ptx::bf16_hi(w0);
+                            sv[j * 8 + 2] = ptx::bf16_lo(w1); sv[j * 8 + 3] = ptx::bf16_hi(w1);
+                            sv[j * 8 + 4] = ptx::bf16_lo(w2); sv[j * 8 + 5] = ptx::bf16_hi(w2);
+                            sv[j * 8 + 6] = ptx::bf16_lo(w3); sv[j * 8 + 7] = ptx::bf16_hi(w3);
+                        }
+                    }
+                    if (EPI == kEpiStoreStats) {
+                        // online softmax statistics of this thread's 32 stored values: running
+                        // maximum st_m and sum of exp(value - st_m), columns >= v_real left out
+                        const int g0 = n0 + col0;
+                        float mx = -INFINITY;
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) {
+                            if (g0 + k >= p.v_real) sv[k] = -INFINITY;
+                            mx = fmaxf(mx, sv[k]);
+                        }
+                        if (mx > st_m) {
+                            st_s *= exp2f((st_m - mx) * 1.4426950408889634f);  // 0 while st_m = -inf
+                            st_m = mx;
+                        }
+                        if (st_m > -INFINITY) {
+                            const float ms = st_m * 1.4426950408889634f;
+                            float acc_s = 0.0f;
+#pragma unroll
+                            for (int k = 0; k < 32; ++k)
+                                acc_s += ptx::ex2_approx(fmaf(sv[k], 1.4426950408889634f, -ms));
+                            st_s += acc_s;
+                        }
                     }
                 } else if (EPI == kEpiSwiglu) {
                     // step c covers out columns [c*64, +64): gate TMEM cols c*64.., up cols 128 + c*64..
@@ -687,20 +730,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
                 // make the staged tile visible to the TMA engine, then one thread stores it
                 ptx::fence_proxy_async_smem();
-                if (leader && SLOTS >= 2) {
+                if (store_warp && SLOTS >= 2) {
                     // the slot the NEXT step writes was last stored SLOTS-1 groups ago
-                    ptx::bulk_wait_group_read<(SLOTS >= 2 ? SLOTS - 2 : 0)>();
+                    if (ptx::elect_one()) ptx::bulk_wait_group_read<(SLOTS >= 2 ? SLOTS - 2 : 0)>();
                 }
                 __syncwarp();
                 ptx::named_bar_sync(1, kEpiThreads);
-                if (leader) {
-                    // The row coordinate is handed to the TMA unit through a fresh register. Without
-                    // this the pair build of the plain-store epilogue issued every store at row 0
-                    // (the long-lived copy of m0 the compiler kept was stale at this point); the
-                    // parity tests on multi-tile shapes guard this.
-                    const int y = ptx::fresh(m0);
+                if (store_warp) {
+                  if (ptx::elect_one()) {
+                    const int y = m0;
                     if (ok && y < p.M) {
-                        if (EPI == kEpiStore || EPI == kEpiMulGeluGrad) {
+                        if (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiMulGeluGrad) {
                             const int x = n0 + c * 64;
                             if (x < p.N) ptx::tma_store_2d(&tmD, buf, x, y);
                         } else if (EPI == kEpiGelu) {
@@ -728,16 +768,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     // every thread has read this step's pre-activation buffer (barrier above): refill it
                     if (EPI == kEpiMulGeluGrad) issue_aux(gstep + AUX_AHEAD);
                     if (SLOTS == 1) ptx::bulk_wait_group_read<0>();
+                  }
                 }
                 __syncwarp();  // the single-lane block above rejoins its warp before collective ops
                 if (SLOTS == 1) ptx::named_bar_sync(1, kEpiThreads);
+            }
+            if (EPI == kEpiStoreStats) {
+                const long long grow = static_cast<long long>(m0) + row;
+                if (ok && grow < p.M)
+                    p.stats[grow * p.stats_ld + n_blk * 2 + hf] = make_float2(st_m, st_s);
             }
             if (++acc == 2) {
                 acc = 0;
                 acc_phase ^= 1u;
             }
         }
-        if (leader) ptx::bulk_wait_group<0>();  // all stores have reached global memory
+        if (store_warp) {
+            if (ptx::elect_one()) ptx::bulk_wait_group<0>();  // all stores have reached global memory
+        }
     }
 
     // ---------------------------------------------------------------- common exit

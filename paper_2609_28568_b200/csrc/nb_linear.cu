@@ -182,6 +182,9 @@ struct GemmArgs {
     int reduce;
     int splits;
     float *dbias;  // wgrad: bias gradient fused into the pass over dz, or null
+    float2 *stats; // forward with softmax statistics: [M, stats_ld]
+    int stats_ld;
+    int v_real;
 };
 
 template <class Cfg>
@@ -247,6 +250,9 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     p.reduce = a.reduce;
     p.bias = static_cast<const __nv_bfloat16 *>(a.bias);
     p.dbias = a.dbias;
+    p.stats = a.stats;
+    p.stats_ld = a.stats_ld;
+    p.v_real = a.v_real;
     p.status = s.status;
     p.timeout_ns = kDefaultTimeoutNs;
     const long long units = 1ll * p.tiles_m * p.tiles_n * p.splits;
@@ -285,6 +291,8 @@ using DgradMulGelu1 = GemmCfg<1, 256, 2, 2, false, true, kEpiMulGeluGrad>;
 using WgradF32_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32>;
 using WgradBf16_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiStore>;
 using FwdStore2 = GemmCfg<2, 256, 6, 2, false, false, kEpiStore>;
+using FwdStoreStats1 = GemmCfg<1, 256, 4, 2, false, false, kEpiStoreStats>;
+using FwdStoreStats2 = GemmCfg<2, 256, 6, 2, false, false, kEpiStoreStats>;
 using FwdGelu2 = GemmCfg<2, 256, 5, 4, false, false, kEpiGelu>;
 using FwdSwiglu2 = GemmCfg<2, 256, 5, 3, false, false, kEpiSwiglu>;
 using DgradStore2 = GemmCfg<2, 256, 6, 2, false, true, kEpiStore>;
@@ -593,6 +601,69 @@ int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int a
     int rc = get_state(&s);
     if (rc != NB_OK) return rc;
     return launch_dbias(*s, static_cast<float *>(dbias), dout, BT, OC, accumulate, g_stream);
+}
+
+int nb_lm_head_ce_forward(void *logits, void *loss, void *lse, const void *inp, const void *weight,
+                          const void *targets, int64_t BT, int64_t C, int64_t Vp, int64_t V,
+                          void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, Vp);
+    if (rc != NB_OK) return rc;
+    if (V <= 0 || V > Vp) return fail(NB_ERR_INVALID_ARG, "V must be within (0, Vp]");
+    if (!logits || !loss || !lse || !inp || !weight || !targets)
+        return fail(NB_ERR_INVALID_ARG, "all pointers must be given");
+    if (!aligned16(logits) || !aligned16(inp) || !aligned16(weight) ||
+        (reinterpret_cast<uintptr_t>(loss) & 3u) || (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+        (reinterpret_cast<uintptr_t>(targets) & 3u))
+        return fail(NB_ERR_INVALID_ARG, "misaligned pointer");
+    if (BT == 0) return NB_OK;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    const int stats_ld = 2 * static_cast<int>((Vp + 255) / 256);
+    if ((rc = ensure_workspace(*s, static_cast<size_t>(BT) * stats_ld * sizeof(float2))) != NB_OK) return rc;
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = weight; a.b_rows = Vp; a.b_cols = C;
+    a.D = logits; a.d_rows = BT; a.d_cols = Vp; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(Vp); a.K = static_cast<int>(C);
+    a.splits = 1;
+    a.stats = static_cast<float2 *>(s->workspace);
+    a.stats_ld = stats_ld;
+    a.v_real = static_cast<int>(V);
+    if ((rc = launch_gemm_auto<FwdStoreStats1, FwdStoreStats2>(*s, a, stream)) != NB_OK) return rc;
+    const unsigned blocks = static_cast<unsigned>((BT + 7) / 8);
+    ce_reduce_kernel<<<blocks, 256, 0, stream>>>(static_cast<float *>(loss), static_cast<float *>(lse),
+                                                 static_cast<const float2 *>(s->workspace), stats_ld,
+                                                 static_cast<const __nv_bfloat16 *>(logits), Vp,
+                                                 static_cast<const int *>(targets), BT, static_cast<int>(V));
+    NB_CUDA(cudaGetLastError());
+    ++g_launches;
+    return NB_OK;
+}
+
+int nb_ce_backward(void *dlogits, const void *logits, const void *lse, const void *targets, float gscale,
+                   int64_t BT, int64_t Vp, int64_t V, void *stream_)
+{
+    if (BT < 0 || Vp <= 0 || V <= 0 || V > Vp) return fail(NB_ERR_INVALID_ARG, "bad dimension");
+    if (Vp % 8 != 0) return fail(NB_ERR_UNSUPPORTED, "Vp must be a multiple of 8");
+    if (BT >= (1ll << 31) || Vp >= (1ll << 31)) return fail(NB_ERR_UNSUPPORTED, "dimension too large");
+    if (!dlogits || !logits || !lse || !targets) return fail(NB_ERR_INVALID_ARG, "all pointers must be given");
+    if (!aligned16(dlogits) || !aligned16(logits)) return fail(NB_ERR_INVALID_ARG, "misaligned pointer");
+    if (BT == 0) return NB_OK;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    const int vec_per_row = static_cast<int>(Vp / 8);
+    ce_backward_kernel<<<elementwise_grid(*s, BT * vec_per_row), 256, 0, static_cast<cudaStream_t>(stream_)>>>(
+        static_cast<uint4 *>(dlogits), static_cast<const uint4 *>(logits), static_cast<const float *>(lse),
+        static_cast<const int *>(targets), gscale, BT, vec_per_row, static_cast<int>(V));
+    NB_CUDA(cudaGetLastError());
+    ++g_launches;
+    return NB_OK;
 }
 
 int nb_cast_f32_to_bf16(void *dst, const void *src, int64_t n, void *stream_)

@@ -318,14 +318,6 @@ __device__ __forceinline__ void st_shared_u32_volatile(uint32_t addr, uint32_t v
     asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-// A value copied through an opaque move: the result lives in a fresh general register, whatever
-// the compiler knew about (or did with) the source.
-__device__ __forceinline__ int fresh(int v)
-{
-    asm volatile("mov.b32 %0, %0;" : "+r"(v));
-    return v;
-}
-
 // ------------------------------------------------------------------ packed fp32 math (two lanes)
 // sm_100 executes fma / mul / add on pairs of fp32 held in a 64-bit register: half the issue slots
 // of the scalar forms, which is what the activation epilogues are short of.
@@ -372,6 +364,12 @@ __device__ __forceinline__ float tanh_approx(float x)
 {
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)

@@ -5,7 +5,8 @@
 KIND: fwd, fwd_nobias, fwd_gelu, fwd_swiglu, dgrad, dgrad_fused (dgrad with the producer's GELU
 backward in the epilogue), wgrad (accumulating), wgrad_bias (wgrad with the fused bias gradient),
 dbias (stand-alone column reduction), bwd (dgrad + wgrad + dbias in one call), cast (fp32 -> bf16
-master-weight cast of OC*C elements; reports GB/s as "TFLOP/s"-free line).
+master-weight cast of OC*C elements; reports GB/s), head_ce (head forward with the fused softmax
+statistics, vocabulary OC with the last 47 columns as padding), ce_bwd (dlogits from logits, GB/s).
 Prints microseconds per call and TFLOP/s from CUDA events around REPS back-to-back calls.
 """
 from __future__ import annotations
@@ -55,6 +56,15 @@ def main(argv) -> int:
         src = torch.randn(n, dtype=f32, device=dev)
         dst = torch.empty(n, dtype=bf, device=dev)
         calls["cast"] = lambda: nb.nb_cast_f32_to_bf16(dst, src, n)
+    if kind in ("head_ce", "ce_bwd"):
+        V = OC - 47 if OC > 47 else OC
+        tg = torch.randint(0, V, (BT,), dtype=torch.int32, device=dev)
+        loss = torch.empty(BT, dtype=f32, device=dev)
+        lse = torch.empty(BT, dtype=f32, device=dev)
+        calls["head_ce"] = lambda: nb.nb_lm_head_ce_forward(out, loss, lse, inp, w, tg, BT, C, OC, V)
+        if kind == "ce_bwd":
+            calls["head_ce"]()
+            calls["ce_bwd"] = lambda: nb.nb_ce_backward(pre, out, lse, tg, 1.0 / BT, BT, OC, V)
     if kind not in calls:
         print(__doc__)
         return 2
@@ -72,6 +82,9 @@ def main(argv) -> int:
     ms = e0.elapsed_time(e1) / reps
     if kind == "cast":
         print(f"cast n={OC * C}: {ms * 1e3:.1f} us/call  {OC * C * 6 / ms / 1e6:.1f} GB/s")
+        return 0
+    if kind == "ce_bwd":
+        print(f"ce_bwd BT={BT} Vp={OC}: {ms * 1e3:.1f} us/call  {BT * OC * 4 / ms / 1e6:.1f} GB/s")
         return 0
     flops = 2 * BT * C * OC * (2 if kind == "bwd" else 1)
     print(f"{kind} BT={BT} C={C} OC={OC}: {ms * 1e3:.1f} us/call  {flops / ms / 1e9:.1f} TFLOP/s")

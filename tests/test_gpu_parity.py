@@ -1,5 +1,7 @@
 """GPU-vs-oracle parity through the C ABI: every element on small and odd shapes and on the
 two small workloads; sampled rows, columns and elements at the full-size workloads."""
+import math
+
 import numpy as np
 import pytest
 import torch
@@ -459,3 +461,68 @@ def test_master_weight_cast_bit_exact():
         assert np.array_equal(got, oracle.cast_f32_bf16(x.numpy())), n
         if dst:
             dst.check("cast")
+
+
+# --------------------------------------------------------------------------- head + cross-entropy
+
+def _ce_case(BT, C, Vp, V, seed, full=True):
+    inp = gen(seed, (BT, C), 1.0)
+    w = gen(seed + 1, (Vp, C), 0.02 if full else 0.05)
+    if V < Vp:
+        w[V:].zero_()
+    g = torch.Generator().manual_seed(seed)
+    targets = torch.randint(0, V, (BT,), generator=g, dtype=torch.int32).to(DEV)
+    logits = Guarded((BT, Vp), torch.bfloat16)
+    loss = Guarded((BT,), torch.float32)
+    lse = Guarded((BT,), torch.float32)
+    nb.nb_lm_head_ce_forward(logits.t, loss.t, lse.t, inp, w, targets, BT, C, Vp, V)
+    ref_logits, _ = nb.linear_forward(inp, w, None, nb.ACT_NONE)
+    assert torch.equal(logits.t, ref_logits)  # the statistics ride along: same logits, bit for bit
+    for gbuf in (logits, loss, lse):
+        gbuf.check("ce forward")
+    return inp, w, targets, logits.t, loss.t, lse.t
+
+
+@pytest.mark.parametrize("BT,C,Vp,V", [(1, 8, 16, 11), (136, 72, 520, 517), (300, 328, 1040, 1000),
+                                        (512, 768, 5120, 5000)])
+def test_head_cross_entropy_small_every_element(BT, C, Vp, V):
+    inp, w, targets, logits, loss, lse = _ce_case(BT, C, Vp, V, 600 + BT, full=False)
+    l_ref, lse_ref, d_ref = oracle.cross_entropy(f32(logits), targets.cpu().numpy(), V, 1.0 / BT)
+    assert np.max(np.abs(f32(lse) - lse_ref)) < 2e-4 * np.max(np.abs(lse_ref)) + 1e-4
+    assert np.max(np.abs(f32(loss) - l_ref)) < 2e-4 * np.max(np.abs(lse_ref)) + 1e-4
+    for in_place in (False, True):
+        src = logits.clone()
+        dl = src if in_place else torch.empty_like(src)
+        nb.nb_ce_backward(dl, src, lse, targets, 1.0 / BT, BT, Vp, V)
+        assert torch.all(dl[:, V:] == 0)  # padding: exactly no gradient
+        check_bf16(dl, d_ref, "dlogits")
+    # an out-of-range target is loud, not silent
+    bad = targets.clone()
+    bad[0] = V
+    loss2 = torch.zeros_like(loss)
+    nb.nb_lm_head_ce_forward(logits, loss2, lse, inp, w, bad, BT, C, Vp, V)
+    assert torch.isnan(loss2[0]) and not torch.isnan(loss2[1:]).any()
+
+
+def test_head_cross_entropy_full_size_sampled():
+    """B=16, T=1024 micro-batch on the padded vocabulary: losses of every row against the oracle on
+    sampled rows, the gradient on sampled rows, and the chain into the head's backward."""
+    BT, C, Vp, V = 16384, 768, shapes.VOCAB_PADDED, shapes.VOCAB_REAL
+    inp, w, targets, logits, loss, lse = _ce_case(BT, C, Vp, V, 700)
+    rows = sample_indices(BT, 48, 701)
+    rt = torch.as_tensor(rows, device=DEV)
+    gscale = 1.0 / BT
+    l_ref, lse_ref, d_ref = oracle.cross_entropy(f32(logits[rt]), targets[rt].cpu().numpy(), V, gscale)
+    assert np.max(np.abs(f32(lse[rt]) - lse_ref)) < 1e-3
+    assert np.max(np.abs(f32(loss[rt]) - l_ref)) < 1e-3
+    # logits ~ N(0, C * 0.02^2): the expected loss at initialisation is log V + variance / 2
+    assert abs(float(loss.mean()) - (math.log(V) + 0.5 * C * 0.02 ** 2)) < 0.02
+    dl = torch.empty_like(logits)
+    nb.nb_ce_backward(dl, logits, lse, targets, gscale, BT, Vp, V)
+    assert torch.all(dl[:, V:] == 0)
+    check_bf16(dl[rt], d_ref, "dlogits rows")
+    rowsum = dl.float().sum(1)
+    assert float(rowsum.abs().max()) < 2e-2 * gscale  # softmax - onehot sums to ~0 (bf16 rounding)
+    dinp, dw, _ = nb.linear_backward(dl, inp, w, need_dbias=False)
+    assert torch.all(dw[V:] == 0)
+    _bwd_sampled("head after ce", dl, inp, w, dinp, dw, None, seed=702, check_dinp_cols=False)

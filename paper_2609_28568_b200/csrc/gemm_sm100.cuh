@@ -641,11 +641,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         // maximum st_m and sum of exp(value - st_m), columns >= v_real left out
                         const int g0 = n0 + col0;
                         float mx = -INFINITY;
+                        if (g0 + 32 > p.v_real) {  // only the tile that straddles v_real masks
 #pragma unroll
-                        for (int k = 0; k < 32; ++k) {
-                            if (g0 + k >= p.v_real) sv[k] = -INFINITY;
-                            mx = fmaxf(mx, sv[k]);
+                            for (int k = 0; k < 32; ++k)
+                                if (g0 + k >= p.v_real) sv[k] = -INFINITY;
                         }
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, sv[k]);
                         if (mx > st_m) {
                             st_s *= exp2f((st_m - mx) * 1.4426950408889634f);  // 0 while st_m = -inf
                             st_m = mx;

@@ -206,3 +206,42 @@ def cross_entropy(logits, targets, V: int, gscale: float = 1.0, want_grad: bool 
     if rc != 0:
         raise ValueError("oracle cross_entropy rejected the request")
     return loss, lse, dl
+
+
+def lora_forward(inp, W, bias, A, B, scale: float):
+    """``inp @ W.T (+ bias) + scale * (inp @ A.T) @ B.T`` in fp64; A [r, C], B [OC, r]."""
+    inp, W, bias, A, B = _f32c(inp), _f32c(W), _f32c(bias), _f32c(A), _f32c(B)
+    BT, C = inp.shape
+    OC, r = B.shape
+    assert W.shape == (OC, C) and A.shape == (r, C)
+    out = np.empty((BT, OC), dtype=np.float64)
+    fn = _load().nbo_lora_forward_f64
+    fn.restype = ctypes.c_int
+    rc = fn(_p(out), _p(inp), _p(W), _p(bias), _p(A), _p(B), ctypes.c_double(scale), ctypes.c_int64(BT),
+            ctypes.c_int64(C), ctypes.c_int64(OC), ctypes.c_int64(r))
+    if rc != 0:
+        raise ValueError("oracle lora_forward rejected the request")
+    return out
+
+
+def lora_backward(dout, inp, W, A, B, scale: float, dA=None, dB=None, accumulate: bool = False,
+                  want_dinp: bool = True):
+    """Gradients of the adapter layer with W frozen: ``(dinp, dA, dB)`` in fp64."""
+    dout, inp, W, A, B = _f32c(dout), _f32c(inp), _f32c(W), _f32c(A), _f32c(B)
+    BT, C = inp.shape
+    OC, r = B.shape
+    dinp = np.empty((BT, C), dtype=np.float64) if want_dinp else None
+    if dA is None:
+        assert not accumulate
+        dA = np.empty((r, C), dtype=np.float64)
+    if dB is None:
+        assert not accumulate
+        dB = np.empty((OC, r), dtype=np.float64)
+    fn = _load().nbo_lora_backward_f64
+    fn.restype = ctypes.c_int
+    rc = fn(_p(dinp), _p(dA), _p(dB), _p(dout), _p(inp), _p(W), _p(A), _p(B), ctypes.c_double(scale),
+            ctypes.c_int64(BT), ctypes.c_int64(C), ctypes.c_int64(OC), ctypes.c_int64(r),
+            ctypes.c_int(1 if accumulate else 0))
+    if rc != 0:
+        raise ValueError("oracle lora_backward rejected the request")
+    return dinp, dA, dB

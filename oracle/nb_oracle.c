@@ -117,6 +117,92 @@ int nbo_cross_entropy_f64(double *loss, double *lse, double *dlogits, const floa
     return 0;
 }
 
+/*
+ * Low-rank adapter beside a frozen linear layer (paper: Method/The clinical stage: rank-16
+ * adapters, rank-stabilised scaling, on the projections of Qwen3-0.6B; base weights frozen).
+ *   t        = inp . A^T                                  [BT, r]      A: [r, C]
+ *   out      = inp . W^T (+ b) + scale * t . B^T          [BT, OC]     B: [OC, r]
+ *   u        = dout . B                                   [BT, r]
+ *   dinp     = dout . W + scale * u . A                   [BT, C]
+ *   dA (+)=    scale * u^T . inp                          [r, C]
+ *   dB (+)=    scale * dout^T . t                         [OC, r]
+ * Intermediates t and u are kept unrounded. Any output pointer may be NULL.
+ */
+int nbo_lora_forward_f64(double *out, const float *inp, const float *W, const float *bias,
+                         const float *A, const float *B, double scale, int64_t BT, int64_t C,
+                         int64_t OC, int64_t r)
+{
+    if (!out || !inp || !W || !A || !B || BT < 0 || C <= 0 || OC <= 0 || r <= 0) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < BT; ++m) {
+        double t[256];
+        for (int64_t j = 0; j < r && j < 256; ++j) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < C; ++k) acc += (double)inp[m * C + k] * (double)A[j * C + k];
+            t[j] = acc;
+        }
+        for (int64_t o = 0; o < OC; ++o) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < C; ++k) acc += (double)inp[m * C + k] * (double)W[o * C + k];
+            if (bias) acc += (double)bias[o];
+            double lo = 0.0;
+            for (int64_t j = 0; j < r; ++j) lo += t[j] * (double)B[o * r + j];
+            out[m * OC + o] = acc + scale * lo;
+        }
+    }
+    return r <= 256 ? 0 : -1;
+}
+
+int nbo_lora_backward_f64(double *dinp, double *dA, double *dB, const float *dout, const float *inp,
+                          const float *W, const float *A, const float *B, double scale, int64_t BT,
+                          int64_t C, int64_t OC, int64_t r, int accumulate)
+{
+    if (!dout || !inp || !W || !A || !B || BT < 0 || C <= 0 || OC <= 0 || r <= 0 || r > 256) return -1;
+    double *t = (double *)malloc(sizeof(double) * (size_t)(BT * r > 0 ? BT * r : 1));
+    double *u = (double *)malloc(sizeof(double) * (size_t)(BT * r > 0 ? BT * r : 1));
+    if (!t || !u) return -2;
+    for (int64_t m = 0; m < BT; ++m)
+        for (int64_t j = 0; j < r; ++j) {
+            double a = 0.0, b = 0.0;
+            for (int64_t k = 0; k < C; ++k) a += (double)inp[m * C + k] * (double)A[j * C + k];
+            for (int64_t o = 0; o < OC; ++o) b += (double)dout[m * OC + o] * (double)B[o * r + j];
+            t[m * r + j] = a;
+            u[m * r + j] = b;
+        }
+    if (dinp) {
+#pragma omp parallel for schedule(static)
+        for (int64_t m = 0; m < BT; ++m)
+            for (int64_t c = 0; c < C; ++c) {
+                double acc = 0.0;
+                for (int64_t o = 0; o < OC; ++o) acc += (double)dout[m * OC + o] * (double)W[o * C + c];
+                double lo = 0.0;
+                for (int64_t j = 0; j < r; ++j) lo += u[m * r + j] * (double)A[j * C + c];
+                dinp[m * C + c] = acc + scale * lo;
+            }
+    }
+    if (dA) {
+        for (int64_t j = 0; j < r; ++j)
+            for (int64_t c = 0; c < C; ++c) {
+                double acc = 0.0;
+                for (int64_t m = 0; m < BT; ++m) acc += u[m * r + j] * (double)inp[m * C + c];
+                if (accumulate) dA[j * C + c] += scale * acc;
+                else dA[j * C + c] = scale * acc;
+            }
+    }
+    if (dB) {
+        for (int64_t o = 0; o < OC; ++o)
+            for (int64_t j = 0; j < r; ++j) {
+                double acc = 0.0;
+                for (int64_t m = 0; m < BT; ++m) acc += (double)dout[m * OC + o] * t[m * r + j];
+                if (accumulate) dB[o * r + j] += scale * acc;
+                else dB[o * r + j] = scale * acc;
+            }
+    }
+    free(t);
+    free(u);
+    return 0;
+}
+
 int nbo_num_threads(void)
 {
 #ifdef _OPENMP

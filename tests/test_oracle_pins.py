@@ -418,3 +418,39 @@ def test_cross_entropy_closed_forms():
     assert np.max(np.abs(l1 - l2)) < 1e-6
     with pytest.raises(ValueError):
         oracle.cross_entropy(a, [0, 1, 2, V], V)
+
+
+# ---------------------------------------------------------------- low-rank adapter beside a frozen layer
+
+def test_lora_against_library_autograd():
+    BT, C, OC, r = 19, 24, 14, 4
+    scale = 32.0 / math.sqrt(16)  # rank-stabilised: alpha / sqrt(r) with the paper's alpha=32, r=16
+    x = _bf16_vals((BT, C), 1.0, 91)
+    W = _bf16_vals((OC, C), 0.3, 92)
+    b = _bf16_vals((OC,), 0.3, 93)
+    A = _bf16_vals((r, C), 0.3, 94)
+    B = _bf16_vals((OC, r), 0.3, 95)
+    dy = _bf16_vals((BT, OC), 1.0, 96)
+    tx = torch.tensor(x, dtype=torch.float64, requires_grad=True)
+    tA = torch.tensor(A, dtype=torch.float64, requires_grad=True)
+    tB = torch.tensor(B, dtype=torch.float64, requires_grad=True)
+    tW = torch.tensor(W, dtype=torch.float64)
+    y = F.linear(tx, tW, torch.tensor(b, dtype=torch.float64)) + scale * F.linear(F.linear(tx, tA), tB)
+    gx, gA, gB = torch.autograd.grad((y * torch.tensor(dy, dtype=torch.float64)).sum(), [tx, tA, tB])
+    out = oracle.lora_forward(x, W, b, A, B, scale)
+    assert np.max(np.abs(out - y.detach().numpy())) < 1e-11
+    dinp, dA, dB = oracle.lora_backward(dy, x, W, A, B, scale)
+    assert np.max(np.abs(dinp - gx.numpy())) < 1e-11
+    assert np.max(np.abs(dA - gA.numpy())) < 1e-11
+    assert np.max(np.abs(dB - gB.numpy())) < 1e-11
+    # B = 0 (the usual initialisation): the layer equals the frozen one and only dB is non-zero
+    Z = np.zeros_like(B)
+    base, _ = oracle.linear_forward(x, W, b)
+    assert np.array_equal(oracle.lora_forward(x, W, b, A, Z, scale), base)
+    dinp0, dA0, dB0 = oracle.lora_backward(dy, x, W, A, Z, scale)
+    assert np.all(dA0 == 0) and np.any(dB0 != 0)
+    assert np.max(np.abs(dinp0 - oracle.linear_backward(dy, x, W, want=("dinp",))["dinp"])) < 1e-12
+    # accumulation over two micro-steps is linear
+    dA2, dB2 = dA.copy(), dB.copy()
+    oracle.lora_backward(dy, x, W, A, B, scale, dA=dA2, dB=dB2, accumulate=True, want_dinp=False)
+    assert np.allclose(dA2, 2 * dA, rtol=1e-14) and np.allclose(dB2, 2 * dB, rtol=1e-14)

@@ -178,6 +178,35 @@ int nb_ce_backward(void *dlogits, const void *logits, const void *lse, const voi
                    float gscale, int64_t BT, int64_t Vp, int64_t V, void *stream);
 
 /*
+ * Low-rank adapter beside a frozen linear layer (paper: Method/The clinical stage: rank-16
+ * adapters with rank-stabilised scaling on the projections of Qwen3-0.6B, base weights frozen).
+ *
+ * nb_lora_linear_forward:
+ *     t   = bf16( scale * inp . lora_a^T )                      [BT, r]   lora_a [r, C]
+ *     out = inp . weight^T (+ bias) + t . lora_b^T              [BT, OC]  lora_b [OC, r]
+ * The second line is ONE GEMM: the r columns of t and lora_b are appended to the K range of the
+ * base product, so the adapter costs one extra k-block in the accumulator, no extra pass over out.
+ * t is an output (bf16, kept for backward). scale is alpha / sqrt(r) (rank-stabilised) or
+ * alpha / r; r a multiple of 8 in [8, 64].
+ *
+ * nb_lora_linear_backward (weight frozen: no dweight):
+ *     u       = bf16( scale * dout . lora_b )                   [BT, r]   caller-provided scratch
+ *     dinp    = dout . weight + u . lora_a                      [BT, C]   one GEMM, K extended by r
+ *     dlora_b (+)= dout^T . t                                   [OC, r]   fp32
+ *     dlora_a (+)= u^T . inp                                    [r, C]    fp32
+ * dinp, dlora_a, dlora_b may be NULL (skipped); accumulate as in nb_linear_backward. t and u are
+ * rounded to bf16 once each (they are tensor-core operands); everything else follows the
+ * conventions at the top of this file.
+ */
+int nb_lora_linear_forward(void *out, void *t, const void *inp, const void *weight, const void *bias,
+                           const void *lora_a, const void *lora_b, float scale, int64_t BT,
+                           int64_t C, int64_t OC, int64_t r, void *stream);
+int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, const void *dout,
+                            const void *inp, const void *weight, const void *lora_a,
+                            const void *lora_b, const void *t, float scale, int64_t BT, int64_t C,
+                            int64_t OC, int64_t r, int accumulate, void *stream);
+
+/*
  * Master-weight cast: dst[i] = bf16(src[i]), round to nearest even, for n elements.
  * (paper: Method/Optimisation and precision keeps fp32 master weights and bf16 compute copies;
  * Results/Speed, the table of levers: the cast is done once per optimizer step and reused by

@@ -24,6 +24,7 @@ EXPORTS = (
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
     "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
     "nb_debug_split_plan", "nb_cast_f32_to_bf16", "nb_lm_head_ce_forward", "nb_ce_backward",
+    "nb_lora_linear_forward", "nb_lora_linear_backward",
 )
 
 _lib = None
@@ -61,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.nb_kernel_launches.restype = _i64
         L.nb_gelu_dbias_noalloc.argtypes = [_vp, _vp, _vp, _i64, _i64, _int, _vp]
         L.nb_cast_f32_to_bf16.argtypes = [_vp, _vp, _i64, _vp]
+        L.nb_lora_linear_forward.argtypes = [_vp] * 7 + [ctypes.c_float] + [_i64] * 4 + [_vp]
+        L.nb_lora_linear_backward.argtypes = [_vp] * 10 + [ctypes.c_float] + [_i64] * 4 + [_int, _vp]
         L.nb_lm_head_ce_forward.argtypes = [_vp] * 6 + [_i64] * 4 + [_vp]
         L.nb_ce_backward.argtypes = [_vp] * 4 + [ctypes.c_float] + [_i64] * 3 + [_vp]
         L.nb_debug_split_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int)]
@@ -153,6 +156,22 @@ def nb_gelu_dbias_noalloc(dbias, dout, pre_act, BT, OC, accumulate, stream=None)
     the library: for callers that may not allocate device memory. BT*OC <= NOALLOC_MAX_ELEMS."""
     _check(lib().nb_gelu_dbias_noalloc(_ptr(dbias), _ptr(dout), _ptr(pre_act), BT, OC,
                                        int(accumulate), _stream() if stream is None else stream))
+
+
+def nb_lora_linear_forward(out, t, inp, weight, bias, lora_a, lora_b, scale, BT, C, OC, r, stream=None) -> None:
+    """out = inp @ W.T (+ bias) + t @ B.T with t = bf16(scale * inp @ A.T), the adapter term fused in."""
+    _check(lib().nb_lora_linear_forward(_ptr(out), _ptr(t), _ptr(inp), _ptr(weight), _ptr(bias),
+                                        _ptr(lora_a), _ptr(lora_b), scale, BT, C, OC, r,
+                                        _stream() if stream is None else stream))
+
+
+def nb_lora_linear_backward(dinp, dlora_a, dlora_b, u, dout, inp, weight, lora_a, lora_b, t, scale, BT, C,
+                            OC, r, accumulate, stream=None) -> None:
+    """Gradients of the adapter layer with the base weight frozen (dinp, dA, dB)."""
+    _check(lib().nb_lora_linear_backward(_ptr(dinp), _ptr(dlora_a), _ptr(dlora_b), _ptr(u), _ptr(dout),
+                                         _ptr(inp), _ptr(weight), _ptr(lora_a), _ptr(lora_b), _ptr(t),
+                                         scale, BT, C, OC, r, int(accumulate),
+                                         _stream() if stream is None else stream))
 
 
 def nb_lm_head_ce_forward(logits, loss, lse, inp, weight, targets, BT, C, Vp, V, stream=None) -> None:

@@ -55,6 +55,9 @@ struct GemmParams {
     int splits;             // split-K factor (kEpiF32), else 1
     int kblocks_per_split;  // 64-wide k blocks handled by one unit
     int kblocks;            // ceil(K / 64)
+    int kblocks_ext;        // extra k-blocks read through the second pair of tensor maps (A2, B2):
+                            // D += A2 . B2^T, the low-rank adapter term; only with splits == 1
+    float alpha;            // kEpiStore family: D = alpha * acc + bias
     int group_m;            // rasterisation: m-tiles per group
     int swiglu_h;           // kEpiSwiglu: H (gate rows [0,H), up rows [H,2H) of B)
     int reduce;             // kEpiF32: 1 reduce-add into D, 0 overwrite
@@ -250,6 +253,7 @@ template <class Cfg>
 __global__ void __launch_bounds__(Cfg::THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmE,
+            const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
             const GemmParams p)
 {
     constexpr int BLOCK_N = Cfg::BLOCK_N;
@@ -343,7 +347,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const int kb0 = split * p.kblocks_per_split;
                 const int kb1 = min(kb0 + p.kblocks_per_split, p.kblocks);
                 const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
-                for (int kb = kb0; kb < kb1; ++kb) {
+                const int kb_end = kb1 + p.kblocks_ext;  // the adapter term's k-blocks come last
+                for (int kb = kb0; kb < kb_end; ++kb) {
+                    const bool ext = kb >= kb1;
+                    const CUtensorMap *mapA = ext ? &tmA2 : &tmA;
+                    const CUtensorMap *mapB = ext ? &tmB2 : &tmB;
                     ok = wait_barrier(wctx, Cfg::DBIAS ? free_bar(stage) : empty_bar(stage), phase ^ 1u,
                                       100 + stage);
                     if (!ok) break;
@@ -352,37 +360,37 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     if (rank == 0) ptx::mbar_expect_tx(full_bar(stage), CG * (Cfg::A_BYTES + Cfg::B_BYTES));
                     const uint32_t sa = smem + Cfg::OFF_A + stage * Cfg::A_BYTES;
                     const uint32_t sb = smem + Cfg::OFF_B + stage * Cfg::B_BYTES;
-                    const int k0 = kb * kBlockK;
+                    const int k0 = (ext ? kb - kb1 : kb) * kBlockK;
                     if (Cfg::A_MN) {  // tensor [K rows, M cols]: boxes of 64(m) x 64(k)
 #pragma unroll
                         for (int j = 0; j < kBlockM / 64; ++j)
-                            load(sa + j * 8192u, &tmA, fb, m0 + j * 64, k0);
+                            load(sa + j * 8192u, mapA, fb, m0 + j * 64, k0);
                     } else {          // tensor [M rows, K cols]: boxes of 64(k) x 64(m)
 #pragma unroll
                         for (int j = 0; j < kBlockM / 64; ++j)
-                            load(sa + j * 8192u, &tmA, fb, k0, m0 + j * 64);
+                            load(sa + j * 8192u, mapA, fb, k0, m0 + j * 64);
                     }
                     // this CTA's share of B's N extent: all of it, or its half of the pair's tile
                     if (Cfg::B_MN) {
                         const int n0 = n_blk * BLOCK_N + static_cast<int>(rank) * Cfg::B_ROWS;
 #pragma unroll
                         for (int j = 0; j < Cfg::B_ROWS / 64; ++j)
-                            load(sb + j * 8192u, &tmB, fb, n0 + j * 64, k0);
+                            load(sb + j * 8192u, mapB, fb, n0 + j * 64, k0);
                     } else if (EPI == kEpiSwiglu) {  // 128 gate rows, then the matching 128 up rows
                         const int n0 = n_blk * 128;
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
                             if (CG == 1 || rank == 0)
-                                load(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
+                                load(sb + j * 8192u, mapB, fb, k0, n0 + j * 64);
                             if (CG == 1 || rank == 1)
-                                load(sb + (CG == 1 ? 16384u : 0u) + j * 8192u, &tmB, fb, k0,
+                                load(sb + (CG == 1 ? 16384u : 0u) + j * 8192u, mapB, fb, k0,
                                      p.swiglu_h + n0 + j * 64);
                         }
                     } else {                          // boxes of 64(k) x 64(n)
                         const int n0 = n_blk * BLOCK_N + static_cast<int>(rank) * Cfg::B_ROWS;
 #pragma unroll
                         for (int j = 0; j < Cfg::B_ROWS / 64; ++j)
-                            load(sb + j * 8192u, &tmB, fb, k0, n0 + j * 64);
+                            load(sb + j * 8192u, mapB, fb, k0, n0 + j * 64);
                     }
                     if (++stage == STAGES) {
                         stage = 0;
@@ -409,7 +417,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (!ok) break;
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BLOCK_N);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                const int kb_end = kb1 + p.kblocks_ext;
+                for (int kb = kb0; kb < kb_end; ++kb) {
                     ok = wait_barrier(wctx, full_bar(stage), phase, 300 + stage);
                     if (!ok) break;
                     ptx::tc_fence_after();
@@ -615,10 +624,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         ptx::ld_shared_f32x4(bias_s + 4u * (col0 + j * 8), b0);
                         ptx::ld_shared_f32x4(bias_s + 4u * (col0 + j * 8 + 4), b1);
                         ptx::f2 z[4];  // eight columns as four packed pairs
-                        z[0] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 0], r[j * 8 + 1]), ptx::make_f2(b0.x, b0.y));
-                        z[1] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 2], r[j * 8 + 3]), ptx::make_f2(b0.z, b0.w));
-                        z[2] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 4], r[j * 8 + 5]), ptx::make_f2(b1.x, b1.y));
-                        z[3] = ptx::add2(ptx::make_f2_bits(r[j * 8 + 6], r[j * 8 + 7]), ptx::make_f2(b1.z, b1.w));
+                        const ptx::f2 al = ptx::make_f2(p.alpha, p.alpha);
+                        z[0] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 0], r[j * 8 + 1]), al, ptx::make_f2(b0.x, b0.y));
+                        z[1] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 2], r[j * 8 + 3]), al, ptx::make_f2(b0.z, b0.w));
+                        z[2] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 4], r[j * 8 + 5]), al, ptx::make_f2(b1.x, b1.y));
+                        z[3] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 6], r[j * 8 + 7]), al, ptx::make_f2(b1.z, b1.w));
                         const uint32_t pos = chunk_pos(hf * 4 + j);
                         if (EPI == kEpiGelu) {
                             ptx::st_shared_v4(buf + kStgBytes + pos, pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),

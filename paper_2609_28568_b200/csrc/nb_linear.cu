@@ -182,6 +182,11 @@ struct GemmArgs {
     int reduce;
     int splits;
     float *dbias;  // wgrad: bias gradient fused into the pass over dz, or null
+    // adapter term D += A2 . B2^T over k2 columns (k2 <= 64), read after the main k range
+    const void *A2; uint64_t a2_rows, a2_cols;
+    const void *B2; uint64_t b2_rows, b2_cols;
+    int k2;
+    float alpha;   // D = alpha * acc (+ bias); 0 is read as 1
     float2 *stats; // forward with softmax statistics: [M, stats_ld]
     int stats_ld;
     int v_real;
@@ -228,6 +233,11 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     } else {
         tE = tD;
     }
+    CUtensorMap tA2 = tA, tB2 = tB;
+    if (a.A2 && a.B2 && a.k2 > 0) {
+        if ((rc = get_tmap(s, &tA2, a.A2, a.a2_rows, a.a2_cols, 0, 64)) != NB_OK) return rc;
+        if ((rc = get_tmap(s, &tB2, a.B2, a.b2_rows, a.b2_cols, 0, 64)) != NB_OK) return rc;
+    }
     GemmParams p;
     memset(&p, 0, sizeof(p));
     p.M = a.M;
@@ -245,6 +255,8 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     // rasterisation: units walk `group_m` row tiles for each column tile before moving to the next
     // column tile. Many column tiles (the head): a tall group keeps the weight tiles' reuse in L2;
     // few column tiles: a short group keeps the row tiles' (measured on B200, 1-2 % either way)
+    p.kblocks_ext = (a.A2 && a.B2 && a.k2 > 0 && p.splits == 1) ? (a.k2 + kBlockK - 1) / kBlockK : 0;
+    p.alpha = a.alpha == 0.0f ? 1.0f : a.alpha;
     p.group_m = (p.tiles_n >= 64 ? 64 : p.tiles_n <= 4 ? 4 : 16) / Cfg::CG;
     p.swiglu_h = a.swiglu_h;
     p.reduce = a.reduce;
@@ -275,7 +287,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     attrs[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
     cfg.numAttrs = g_use_pdl ? 2 : 1;
-    NB_CUDA(cudaLaunchKernelEx(&cfg, gemm_kernel<Cfg>, tA, tB, tD, tE, p));
+    NB_CUDA(cudaLaunchKernelEx(&cfg, gemm_kernel<Cfg>, tA, tB, tD, tE, tA2, tB2, p));
     ++g_launches;
     return NB_OK;
 }
@@ -385,6 +397,34 @@ int elementwise_grid(const DeviceState &s, long long nvec)
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     return static_cast<int>(blocks);
+}
+
+// dweight[M_, N_] (+)= dz^T . inp over BT rows, fp32, with the split-K factor chosen per shape;
+// dz [BT, M_], inp [BT, N_]. dbias (or null) is summed inside the same kernel.
+int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight, float *dbias,
+                  int64_t BT, int64_t M_, int64_t N_, int accumulate, cudaStream_t stream)
+{
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = dz; a.a_rows = BT; a.a_cols = M_;
+    a.B = inp; a.b_rows = BT; a.b_cols = N_;
+    a.D = dweight; a.d_rows = M_; a.d_cols = N_; a.d_dtype = 1;
+    a.M = static_cast<int>(M_); a.N = static_cast<int>(N_); a.K = static_cast<int>(BT);
+    const int tile_m = use_pairs(a.M) ? 2 * kBlockM : kBlockM;
+    const int tiles = ((a.M + tile_m - 1) / tile_m) * ((a.N + 255) / 256);
+    const int kblocks = (a.K + kBlockK - 1) / kBlockK;
+    const int slots = s.num_sms / (use_pairs(a.M) ? 2 : 1);  // tiles resident at once
+    const int splits = choose_splits(tiles, kblocks, slots);
+    a.splits = splits;
+    a.reduce = (accumulate || splits > 1) ? 1 : 0;
+    if (!accumulate && splits > 1)
+        NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(M_ * N_) * 4, stream));
+    if (dbias) {  // the bias gradient rides along: reducer warps sum dz while it is in shared memory
+        if (!accumulate) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(M_) * 4, stream));
+        a.dbias = dbias;
+        return launch_gemm_auto<WgradF32Bias1, WgradF32Bias2>(s, a, stream);
+    }
+    return launch_gemm_auto<WgradF32_1, WgradF32_2>(s, a, stream);
 }
 
 }  // namespace
@@ -547,24 +587,9 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
         a.D = dweight; a.d_rows = OC; a.d_cols = C;
         a.M = static_cast<int>(OC); a.N = static_cast<int>(C); a.K = static_cast<int>(BT);
         if (dweight_dtype == NB_DTYPE_F32) {
-            a.d_dtype = 1;
-            const int tile_m = use_pairs(a.M) ? 2 * kBlockM : kBlockM;
-            const int tiles = ((a.M + tile_m - 1) / tile_m) * ((a.N + 255) / 256);
-            const int kblocks = (a.K + kBlockK - 1) / kBlockK;
-            const int slots = s->num_sms / (use_pairs(a.M) ? 2 : 1);  // tiles resident at once
-            const int splits = choose_splits(tiles, kblocks, slots);
-            a.splits = splits;
-            a.reduce = (accumulate || splits > 1) ? 1 : 0;
-            if (!accumulate && splits > 1)
-                NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(OC * C) * 4, stream));
-            if (dbias) {  // the bias gradient rides along: reducer warps sum dz while it is in shared memory
-                if (!accumulate) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
-                a.dbias = static_cast<float *>(dbias);
-                rc = launch_gemm_auto<WgradF32Bias1, WgradF32Bias2>(*s, a, stream);
-                dbias = nullptr;  // done
-            } else {
-                rc = launch_gemm_auto<WgradF32_1, WgradF32_2>(*s, a, stream);
-            }
+            rc = run_wgrad_f32(*s, dz, inp, dweight, static_cast<float *>(dbias), BT, OC, C, accumulate,
+                               stream);
+            dbias = nullptr;  // done inside the wgrad kernel
         } else {
             a.d_dtype = 0;
             a.splits = 1;
@@ -663,6 +688,101 @@ int nb_ce_backward(void *dlogits, const void *logits, const void *lse, const voi
         static_cast<const int *>(targets), gscale, BT, vec_per_row, static_cast<int>(V));
     NB_CUDA(cudaGetLastError());
     ++g_launches;
+    return NB_OK;
+}
+
+int nb_lora_linear_forward(void *out, void *t, const void *inp, const void *weight, const void *bias,
+                           const void *lora_a, const void *lora_b, float scale, int64_t BT, int64_t C,
+                           int64_t OC, int64_t r, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, OC);
+    if (rc != NB_OK) return rc;
+    if (r < 8 || r > 64 || r % 8 != 0) return fail(NB_ERR_UNSUPPORTED, "rank must be 8..64, a multiple of 8");
+    if (!out || !t || !inp || !weight || !lora_a || !lora_b)
+        return fail(NB_ERR_INVALID_ARG, "out, t, inp, weight, lora_a and lora_b must not be NULL");
+    if (!aligned16(out) || !aligned16(t) || !aligned16(inp) || !aligned16(weight) || !aligned16(lora_a) ||
+        !aligned16(lora_b))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (BT == 0) return NB_OK;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));  // t = scale * inp . A^T
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = lora_a; a.b_rows = r; a.b_cols = C;
+    a.D = t; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(C);
+    a.splits = 1;
+    a.alpha = scale;
+    if ((rc = launch_gemm_auto<FwdStore1, FwdStore2>(*s, a, stream)) != NB_OK) return rc;
+    memset(&a, 0, sizeof(a));  // out = inp . W^T (+ bias) + t . B^T: r extra columns of K
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = weight; a.b_rows = OC; a.b_cols = C;
+    a.D = out; a.d_rows = BT; a.d_cols = OC; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(OC); a.K = static_cast<int>(C);
+    a.bias = bias;
+    a.splits = 1;
+    a.A2 = t; a.a2_rows = BT; a.a2_cols = r;
+    a.B2 = lora_b; a.b2_rows = OC; a.b2_cols = r;
+    a.k2 = static_cast<int>(r);
+    return launch_gemm_auto<FwdStore1, FwdStore2>(*s, a, stream);
+}
+
+int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, const void *dout,
+                            const void *inp, const void *weight, const void *lora_a, const void *lora_b,
+                            const void *t, float scale, int64_t BT, int64_t C, int64_t OC, int64_t r,
+                            int accumulate, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, OC);
+    if (rc != NB_OK) return rc;
+    if (r < 8 || r > 64 || r % 8 != 0) return fail(NB_ERR_UNSUPPORTED, "rank must be 8..64, a multiple of 8");
+    if (!u || !dout || !inp || !lora_a || !lora_b)
+        return fail(NB_ERR_INVALID_ARG, "u, dout, inp, lora_a and lora_b must not be NULL");
+    if (dinp && !weight) return fail(NB_ERR_INVALID_ARG, "weight is required to compute dinp");
+    if (dlora_b && !t) return fail(NB_ERR_INVALID_ARG, "t (from the forward call) is required for dlora_b");
+    if (!aligned16(dinp) || !aligned16(dlora_a) || !aligned16(dlora_b) || !aligned16(u) || !aligned16(dout) ||
+        !aligned16(inp) || !aligned16(weight) || !aligned16(lora_a) || !aligned16(lora_b) || !aligned16(t))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    if (BT == 0) {
+        if (!accumulate) {
+            if (dlora_a) NB_CUDA(cudaMemsetAsync(dlora_a, 0, static_cast<size_t>(r * C) * 4, stream));
+            if (dlora_b) NB_CUDA(cudaMemsetAsync(dlora_b, 0, static_cast<size_t>(OC * r) * 4, stream));
+        }
+        return NB_OK;
+    }
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));  // u = scale * dout . B   (B [OC, r] read as an MN-major operand)
+    a.A = dout; a.a_rows = BT; a.a_cols = OC;
+    a.B = lora_b; a.b_rows = OC; a.b_cols = r;
+    a.D = u; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
+    a.splits = 1;
+    a.alpha = scale;
+    if ((rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream)) != NB_OK) return rc;
+    if (dinp) {  // dinp = dout . W + u . A: r extra rows of K
+        memset(&a, 0, sizeof(a));
+        a.A = dout; a.a_rows = BT; a.a_cols = OC;
+        a.B = weight; a.b_rows = OC; a.b_cols = C;
+        a.D = dinp; a.d_rows = BT; a.d_cols = C; a.d_dtype = 0;
+        a.M = static_cast<int>(BT); a.N = static_cast<int>(C); a.K = static_cast<int>(OC);
+        a.splits = 1;
+        a.A2 = u; a.a2_rows = BT; a.a2_cols = r;
+        a.B2 = lora_a; a.b2_rows = r; a.b2_cols = C;
+        a.k2 = static_cast<int>(r);
+        if ((rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream)) != NB_OK) return rc;
+    }
+    if (dlora_b)  // dB [OC, r] (+)= dout^T . t      (t already carries the scale)
+        if ((rc = run_wgrad_f32(*s, dout, t, dlora_b, nullptr, BT, OC, r, accumulate, stream)) != NB_OK)
+            return rc;
+    if (dlora_a)  // dA [r, C] (+)= u^T . inp        (u already carries the scale)
+        if ((rc = run_wgrad_f32(*s, u, inp, dlora_a, nullptr, BT, r, C, accumulate, stream)) != NB_OK)
+            return rc;
     return NB_OK;
 }
 

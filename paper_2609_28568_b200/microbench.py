@@ -6,7 +6,8 @@ KIND: fwd, fwd_nobias, fwd_gelu, fwd_swiglu, dgrad, dgrad_fused (dgrad with the 
 backward in the epilogue), wgrad (accumulating), wgrad_bias (wgrad with the fused bias gradient),
 dbias (stand-alone column reduction), bwd (dgrad + wgrad + dbias in one call), cast (fp32 -> bf16
 master-weight cast of OC*C elements; reports GB/s), head_ce (head forward with the fused softmax
-statistics, vocabulary OC with the last 47 columns as padding), ce_bwd (dlogits from logits, GB/s).
+statistics, vocabulary OC with the last 47 columns as padding), ce_bwd (dlogits from logits, GB/s),
+lora_fwd / lora_bwd (rank-16 adapter beside a frozen weight; TFLOP/s counts base + adapter flops).
 Prints microseconds per call and TFLOP/s from CUDA events around REPS back-to-back calls.
 """
 from __future__ import annotations
@@ -65,6 +66,18 @@ def main(argv) -> int:
         if kind == "ce_bwd":
             calls["head_ce"]()
             calls["ce_bwd"] = lambda: nb.nb_ce_backward(pre, out, lse, tg, 1.0 / BT, BT, OC, V)
+    if kind in ("lora_fwd", "lora_bwd"):
+        r, scale = 16, 8.0
+        la = synth.normal(6, (r, C), 0.02, dev)
+        lb = synth.normal(7, (OC, r), 0.02, dev)
+        t = torch.empty((BT, r), dtype=bf, device=dev)
+        u = torch.empty((BT, r), dtype=bf, device=dev)
+        dla = torch.zeros((r, C), dtype=f32, device=dev)
+        dlb = torch.zeros((OC, r), dtype=f32, device=dev)
+        calls["lora_fwd"] = lambda: nb.nb_lora_linear_forward(out, t, inp, w, None, la, lb, scale, BT, C, OC, r)
+        calls["lora_fwd"]()
+        calls["lora_bwd"] = lambda: nb.nb_lora_linear_backward(dinp, dla, dlb, u, dout, inp, w, la, lb, t,
+                                                               scale, BT, C, OC, r, 1)
     if kind not in calls:
         print(__doc__)
         return 2
@@ -87,6 +100,10 @@ def main(argv) -> int:
         print(f"ce_bwd BT={BT} Vp={OC}: {ms * 1e3:.1f} us/call  {BT * OC * 4 / ms / 1e6:.1f} GB/s")
         return 0
     flops = 2 * BT * C * OC * (2 if kind == "bwd" else 1)
+    if kind == "lora_fwd":
+        flops += 2 * BT * 16 * (C + OC)
+    if kind == "lora_bwd":
+        flops += 4 * BT * 16 * (C + OC)
     print(f"{kind} BT={BT} C={C} OC={OC}: {ms * 1e3:.1f} us/call  {flops / ms / 1e9:.1f} TFLOP/s")
     return 0
 

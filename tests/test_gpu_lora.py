@@ -1,0 +1,168 @@
+"""GPU-vs-oracle parity of the low-rank adapter layer (frozen base weight, rank-r A and B):
+every element on small and odd shapes, sampled rows at the adapter workload's full size."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_28568_b200 import binding as nb
+from paper_2609_28568_b200 import synth
+from parity import Guarded, check_bf16, check_f32, f32, sample_indices
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(autouse=True)
+def _status_clean():
+    yield
+    nb.nb_check_status()
+
+
+def gen(seed, shape, std):
+    return synth.normal(seed, shape, std, DEV)
+
+
+def _rounding_slack(mid_ref, other):
+    """The call rounds its rank-r intermediate (t or u) to bf16 once, a relative error of at most
+    2^-9 per element; through the second factor that moves an output by at most this much."""
+    return 2.0 ** -9 * (np.abs(mid_ref) @ np.abs(np.asarray(other, np.float64)))
+
+
+def _tensors(BT, C, OC, r, bias, seed):
+    inp = gen(seed, (BT, C), 1.0)
+    w = gen(seed + 1, (OC, C), 0.02)
+    b = gen(seed + 2, (OC,), 0.02) if bias else None
+    a = gen(seed + 3, (r, C), 0.02)
+    bb = gen(seed + 4, (OC, r), 0.02)  # a trained adapter: B is no longer zero
+    dout = gen(seed + 5, (BT, OC), 1e-3)
+    return inp, w, b, a, bb, dout
+
+
+@pytest.mark.parametrize("bias", [False, True])
+@pytest.mark.parametrize("BT,C,OC,r", [
+    (1, 8, 8, 8),            # smallest legal problem
+    (200, 72, 136, 16),      # ragged in every dimension, one tile
+    (300, 328, 520, 16),     # several n-tiles, ragged tails, a CTA pair
+    (640, 256, 768, 64),     # the extension fills a whole k-block
+    (520, 1024, 1024, 24),   # many k-blocks before the extension
+])
+def test_adapter_layer_every_element(BT, C, OC, r, bias):
+    scale = 32.0 / math.sqrt(r)  # rank-stabilised scaling
+    inp, w, b, a, bb, dout = _tensors(BT, C, OC, r, bias, seed=900)
+    out = Guarded((BT, OC), torch.bfloat16)
+    t = Guarded((BT, r), torch.bfloat16)
+    nb.nb_lora_linear_forward(out.t, t.t, inp, w, b, a, bb, scale, BT, C, OC, r)
+    o_ref = oracle.lora_forward(f32(inp), f32(w), f32(b) if bias else None, f32(a), f32(bb), scale)
+    t_ref, _ = oracle.linear_forward(f32(inp), f32(a))
+    check_bf16(t.t, scale * t_ref, "t")
+    check_bf16(out.t, o_ref, "out", extra=_rounding_slack(scale * t_ref, f32(bb).T))
+    # and with the stored t as the oracle's input the layer is one product over [inp | t]
+    o_ref2, _ = oracle.linear_forward(np.concatenate([f32(inp), f32(t.t)], axis=1),
+                                      np.concatenate([f32(w), f32(bb)], axis=1), f32(b) if bias else None)
+    check_bf16(out.t, o_ref2, "out from stored t")
+    out.check("out")
+    t.check("t")
+    # the adapter term must be visible in this test, or the comparison proves nothing about it
+    base, _ = oracle.linear_forward(f32(inp), f32(w), f32(b) if bias else None)
+    assert np.abs(o_ref - base).max() > 0.05 * np.abs(base).max()
+
+    dinp = Guarded((BT, C), torch.bfloat16)
+    u = Guarded((BT, r), torch.bfloat16)
+    dA = Guarded((r, C), torch.float32, fill=777.0)   # accumulate=0 must overwrite
+    dB = Guarded((OC, r), torch.float32, fill=-55.0)
+    nb.nb_lora_linear_backward(dinp.t, dA.t, dB.t, u.t, dout, inp, w, a, bb, t.t, scale, BT, C, OC, r, 0)
+    di_ref, dA_ref, dB_ref = oracle.lora_backward(f32(dout), f32(inp), f32(w), f32(a), f32(bb), scale)
+    u_ref = oracle.linear_backward(f32(dout), None, f32(bb), want=("dinp",))["dinp"]
+    check_bf16(u.t, scale * u_ref, "u")
+    check_bf16(dinp.t, di_ref, "dinp", extra=_rounding_slack(scale * u_ref, f32(a)))
+    di_ref2 = oracle.linear_backward(np.concatenate([f32(dout), f32(u.t)], axis=1), None,
+                                     np.concatenate([f32(w), f32(a)], axis=0), want=("dinp",))["dinp"]
+    check_bf16(dinp.t, di_ref2, "dinp from stored u")
+    check_f32(dA.t, dA_ref, "dlora_a")
+    check_f32(dB.t, dB_ref, "dlora_b")
+    for g, n in ((dinp, "dinp"), (u, "u"), (dA, "dlora_a"), (dB, "dlora_b")):
+        g.check(n)
+
+    # a second micro-step accumulates; dinp is skipped
+    dout2 = gen(990, (BT, OC), 1e-3)
+    nb.nb_lora_linear_backward(None, dA.t, dB.t, u.t, dout2, inp, w, a, bb, t.t, scale, BT, C, OC, r, 1)
+    _, dA_ref2, dB_ref2 = oracle.lora_backward(f32(dout2), f32(inp), f32(w), f32(a), f32(bb), scale,
+                                               dA=dA_ref.copy(), dB=dB_ref.copy(), accumulate=True,
+                                               want_dinp=False)
+    check_f32(dA.t, dA_ref2, "dlora_a step 2")
+    check_f32(dB.t, dB_ref2, "dlora_b step 2")
+
+
+def test_zero_b_reduces_to_the_base_layer_bit_for_bit():
+    """A freshly initialised adapter (B = 0) must give exactly the base layer's output and dinp."""
+    BT, C, OC, r = 400, 264, 392, 16
+    inp, w, b, a, _, dout = _tensors(BT, C, OC, r, True, seed=940)
+    zb = torch.zeros((OC, r), dtype=torch.bfloat16, device=DEV)
+    out = torch.empty((BT, OC), dtype=torch.bfloat16, device=DEV)
+    t = torch.empty((BT, r), dtype=torch.bfloat16, device=DEV)
+    nb.nb_lora_linear_forward(out, t, inp, w, b, a, zb, 8.0, BT, C, OC, r)
+    base, _ = nb.linear_forward(inp, w, b, nb.ACT_NONE)
+    assert torch.equal(out, base)
+    dinp = torch.empty((BT, C), dtype=torch.bfloat16, device=DEV)
+    u = torch.empty((BT, r), dtype=torch.bfloat16, device=DEV)
+    dA = torch.empty((r, C), dtype=torch.float32, device=DEV)
+    nb.nb_lora_linear_backward(dinp, dA, None, u, dout, inp, w, a, zb, None, 8.0, BT, C, OC, r, 0)
+    dbase, _, _ = nb.linear_backward(dout, inp, w, need_dweight=False, need_dbias=False)
+    assert torch.equal(dinp, dbase)
+    assert float(u.float().abs().max()) == 0.0 and float(dA.abs().max()) == 0.0
+
+
+def test_adapter_rejects_bad_rank_and_missing_tensors():
+    BT, C, OC = 64, 64, 64
+    x = torch.zeros((BT, C), dtype=torch.bfloat16, device=DEV)
+    w = torch.zeros((OC, C), dtype=torch.bfloat16, device=DEV)
+    for r in (4, 12, 72):
+        a = torch.zeros((r, C), dtype=torch.bfloat16, device=DEV)
+        b = torch.zeros((OC, r), dtype=torch.bfloat16, device=DEV)
+        t = torch.zeros((BT, r), dtype=torch.bfloat16, device=DEV)
+        with pytest.raises(nb.NbError) as e:
+            nb.nb_lora_linear_forward(x, t, x, w, None, a, b, 1.0, BT, C, OC, r)
+        assert e.value.code == nb.NB_ERR_UNSUPPORTED
+    a = torch.zeros((16, C), dtype=torch.bfloat16, device=DEV)
+    b = torch.zeros((OC, 16), dtype=torch.bfloat16, device=DEV)
+    t = torch.zeros((BT, 16), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(nb.NbError) as e:
+        nb.nb_lora_linear_forward(x, None, x, w, None, a, b, 1.0, BT, C, OC, 16)
+    assert e.value.code == nb.NB_ERR_INVALID_ARG
+    dB = torch.zeros((OC, 16), dtype=torch.float32, device=DEV)
+    with pytest.raises(nb.NbError) as e:  # dlora_b needs the forward call's t
+        nb.nb_lora_linear_backward(None, None, dB, t, x, x, w, a, b, None, 1.0, BT, C, OC, 16, 0)
+    assert e.value.code == nb.NB_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("C,OC", [(1024, 2048), (3072, 1024)])
+def test_adapter_workload_full_batch_sampled(C, OC):
+    """Qwen3-0.6B q and down projections with rank-16 adapters at B=8, T=2048."""
+    BT, r = 16384, 16
+    scale = 32.0 / math.sqrt(r)
+    inp, w, _, a, bb, dout = _tensors(BT, C, OC, r, False, seed=960)
+    out = torch.empty((BT, OC), dtype=torch.bfloat16, device=DEV)
+    t = torch.empty((BT, r), dtype=torch.bfloat16, device=DEV)
+    nb.nb_lora_linear_forward(out, t, inp, w, None, a, bb, scale, BT, C, OC, r)
+    dinp = torch.empty((BT, C), dtype=torch.bfloat16, device=DEV)
+    u = torch.empty((BT, r), dtype=torch.bfloat16, device=DEV)
+    dA = torch.empty((r, C), dtype=torch.float32, device=DEV)
+    dB = torch.empty((OC, r), dtype=torch.float32, device=DEV)
+    nb.nb_lora_linear_backward(dinp, dA, dB, u, dout, inp, w, a, bb, t, scale, BT, C, OC, r, 0)
+
+    rows = sample_indices(BT, 64, 961)
+    rt = torch.as_tensor(rows, device=DEV)
+    o_ref = oracle.lora_forward(f32(inp[rt]), f32(w), None, f32(a), f32(bb), scale)
+    t_ref, _ = oracle.linear_forward(f32(inp[rt]), f32(a))
+    check_bf16(out[rt], o_ref, "out rows", extra=_rounding_slack(scale * t_ref, f32(bb).T))
+    di_ref, _, _ = oracle.lora_backward(f32(dout[rt]), f32(inp[rt]), f32(w), f32(a), f32(bb), scale)
+    u_ref = oracle.linear_backward(f32(dout[rt]), None, f32(bb), want=("dinp",))["dinp"]
+    check_bf16(dinp[rt], di_ref, "dinp rows", extra=_rounding_slack(scale * u_ref, f32(a)))
+    # the adapter gradients sum over every row: the oracle runs them in full (they are cheap)
+    _, dA_ref, dB_ref = oracle.lora_backward(f32(dout), f32(inp), f32(w), f32(a), f32(bb), scale,
+                                             want_dinp=False)
+    check_f32(dA, dA_ref, "dlora_a")
+    check_f32(dB, dB_ref, "dlora_b")

@@ -313,6 +313,13 @@ using WgradF32_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32>;
 using WgradF32Bias1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32, true>;
 using WgradF32Bias2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32, true>;
 using WgradBf16_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiStore>;
+// Narrow results (N <= 64: the rank-r products of the adapter layer). A 256-wide tile would spend
+// 4-16x the tensor-core time on padding; a 64-wide one leaves these products bound by the read of
+// their tall operand, so they run one CTA per tile with a deep ring.
+using FwdStoreNarrow = GemmCfg<1, 64, 7, 2, false, false, kEpiStore>;
+using DgradStoreNarrow = GemmCfg<1, 64, 7, 2, false, true, kEpiStore>;
+using WgradF32Narrow = GemmCfg<1, 64, 7, 2, true, true, kEpiF32>;
+constexpr int kNarrowN = 64;
 
 bool use_pairs(int M)
 {
@@ -410,10 +417,13 @@ int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight
     a.B = inp; a.b_rows = BT; a.b_cols = N_;
     a.D = dweight; a.d_rows = M_; a.d_cols = N_; a.d_dtype = 1;
     a.M = static_cast<int>(M_); a.N = static_cast<int>(N_); a.K = static_cast<int>(BT);
-    const int tile_m = use_pairs(a.M) ? 2 * kBlockM : kBlockM;
-    const int tiles = ((a.M + tile_m - 1) / tile_m) * ((a.N + 255) / 256);
+    const bool narrow = dbias == nullptr && a.N <= kNarrowN;
+    const bool pairs = !narrow && use_pairs(a.M);
+    const int tile_m = pairs ? 2 * kBlockM : kBlockM;
+    const int tile_n = narrow ? kNarrowN : 256;
+    const int tiles = ((a.M + tile_m - 1) / tile_m) * ((a.N + tile_n - 1) / tile_n);
     const int kblocks = (a.K + kBlockK - 1) / kBlockK;
-    const int slots = s.num_sms / (use_pairs(a.M) ? 2 : 1);  // tiles resident at once
+    const int slots = s.num_sms / (pairs ? 2 : 1);  // tiles resident at once
     const int splits = choose_splits(tiles, kblocks, slots);
     a.splits = splits;
     a.reduce = (accumulate || splits > 1) ? 1 : 0;
@@ -424,6 +434,7 @@ int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight
         a.dbias = dbias;
         return launch_gemm_auto<WgradF32Bias1, WgradF32Bias2>(s, a, stream);
     }
+    if (narrow) return launch_gemm<WgradF32Narrow>(s, a, stream);
     return launch_gemm_auto<WgradF32_1, WgradF32_2>(s, a, stream);
 }
 
@@ -716,7 +727,7 @@ int nb_lora_linear_forward(void *out, void *t, const void *inp, const void *weig
     a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(C);
     a.splits = 1;
     a.alpha = scale;
-    if ((rc = launch_gemm_auto<FwdStore1, FwdStore2>(*s, a, stream)) != NB_OK) return rc;
+    if ((rc = launch_gemm<FwdStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
     memset(&a, 0, sizeof(a));  // out = inp . W^T (+ bias) + t . B^T: r extra columns of K
     a.A = inp; a.a_rows = BT; a.a_cols = C;
     a.B = weight; a.b_rows = OC; a.b_cols = C;
@@ -764,7 +775,7 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
     a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
     a.splits = 1;
     a.alpha = scale;
-    if ((rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream)) != NB_OK) return rc;
+    if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
     if (dinp) {  // dinp = dout . W + u . A: r extra rows of K
         memset(&a, 0, sizeof(a));
         a.A = dout; a.a_rows = BT; a.a_cols = OC;

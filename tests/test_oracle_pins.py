@@ -443,6 +443,10 @@ def test_lora_against_library_autograd():
     assert np.max(np.abs(dinp - gx.numpy())) < 1e-11
     assert np.max(np.abs(dA - gA.numpy())) < 1e-11
     assert np.max(np.abs(dB - gB.numpy())) < 1e-11
+    # merged-weight identity: the adapter is a rank-r update of W
+    Wm = W.astype(np.float64) + scale * (B.astype(np.float64) @ A.astype(np.float64))
+    assert np.max(np.abs(out - (x.astype(np.float64) @ Wm.T + b))) < 1e-11
+    assert np.max(np.abs(dinp - dy.astype(np.float64) @ Wm)) < 1e-11
     # B = 0 (the usual initialisation): the layer equals the frozen one and only dB is non-zero
     Z = np.zeros_like(B)
     base, _ = oracle.linear_forward(x, W, b)

@@ -96,8 +96,17 @@ struct GemmCfg {
     static constexpr int NAUX = (EPI_ == kEpiMulGeluGrad) ? 4 : 0;
     static constexpr uint32_t OFF_AUX = OFF_STG + NSTG * kStgBytes;
     static constexpr uint32_t OFF_BIAS = OFF_AUX + NAUX * kStgBytes;
-    static constexpr uint32_t OFF_BAR = OFF_BIAS + BLOCK_N * 4;
-    static constexpr uint32_t SMEM_BYTES = OFF_BAR + 256;
+    // Warp-private epilogue (bf16 results of full-width tiles): every epilogue warp stages and
+    // stores its own 32-row boxes, no barrier joins the warps. The bias then lives in two buffers
+    // (by tile parity) and each warp has its own pair of pre-activation barriers.
+    static constexpr bool WARP_EPI = BLOCK_N_ == 256 && !DBIAS_ &&
+                                     (EPI_ == kEpiStore || EPI_ == kEpiStoreStats || EPI_ == kEpiGelu ||
+                                      EPI_ == kEpiMulGeluGrad);
+    static constexpr int OUT_BOX_ROWS = WARP_EPI ? 32 : kBlockM;
+    static constexpr uint32_t BIAS_BYTES = (WARP_EPI ? 2 : 1) * BLOCK_N * 4;
+    static constexpr uint32_t OFF_BAR = OFF_BIAS + BIAS_BYTES;
+    static constexpr uint32_t BAR_BYTES = WARP_EPI ? 512 : 256;
+    static constexpr uint32_t SMEM_BYTES = OFF_BAR + BAR_BYTES;
     static constexpr uint32_t TMEM_COLS = (2 * BLOCK_N <= 32) ? 32
                                           : (2 * BLOCK_N <= 64) ? 64
                                           : (2 * BLOCK_N <= 128) ? 128
@@ -114,6 +123,9 @@ struct GemmCfg {
     static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 2, "staging ring");
     static_assert(EPI != kEpiSwiglu || BLOCK_N == 256, "SwiGLU tiles pair 128 gate + 128 up cols");
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+    static_assert(!WARP_EPI || NSTG * kStgBytes >= 8u * BUFS_PER_STEP * 4096u, "a box per warp and plane");
+    static_assert(!WARP_EPI || EPI_ != kEpiMulGeluGrad || NAUX * kStgBytes >= 8u * 2u * 4096u,
+                  "two pre-activation boxes per warp");
     static_assert(!DBIAS_ || (A_MN_ && EPI_ == kEpiF32), "the fused bias gradient belongs to wgrad");
 };
 
@@ -299,6 +311,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ptx::mbar_init(tempty_bar(b), kEpiWarps * CG);  // one arrive per epilogue warp of the tile
         }
         for (int b = 0; b < 4; ++b) ptx::mbar_init(aux_bar(b), 1);
+        if (Cfg::WARP_EPI && EPI == kEpiMulGeluGrad)  // two per epilogue warp, above the common slots
+            for (int b = 0; b < 2 * kEpiWarps; ++b) ptx::mbar_init(bar0 + 256u + 8u * b, 1);
         ptx::st_shared_u32_volatile(abort_addr, 0);
         ptx::st_shared_u32_volatile(epi_abort_addr, 0);
         ptx::fence_barrier_init();
@@ -524,6 +538,222 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int q = warp & 3;
         const int hf = (warp - 2) >> 2;
         const int row = q * 32 + lane;
+      if constexpr (Cfg::WARP_EPI) {
+        // ------------------------------------------------------------ epilogue, warp by warp
+        // A warp owns 32 rows (its TMEM lane quarter) x 128 columns (its half) of the tile. It reads
+        // them from TMEM 32 columns at a time (the next load in flight while it works on the
+        // current one), applies the epilogue, stages 32 x 64 boxes in its own 4 KB buffers and
+        // stores them with its own TMA copies. No barrier joins the warps: while one waits for
+        // TMEM, a proxy fence or a store, the others compute.
+        const int ew = warp - 2;                  // 0..7
+        constexpr uint32_t kBoxBytes = 32 * 128;  // 32 rows x 64 bf16, 128-byte swizzled
+        constexpr uint32_t NBUF = Cfg::BUFS_PER_STEP;  // 1; kEpiGelu: activated + pre-activation
+        const uint32_t stg = smem + Cfg::OFF_STG + static_cast<uint32_t>(ew) * NBUF * kBoxBytes;
+        const uint32_t aux0 = smem + Cfg::OFF_AUX + static_cast<uint32_t>(ew) * 2u * kBoxBytes;
+        const uint32_t lane_off = static_cast<uint32_t>(lane) * 128u;
+        const uint32_t sw = static_cast<uint32_t>(lane & 7);
+        auto chunk_pos = [&](int chunk) { return lane_off + ((static_cast<uint32_t>(chunk) ^ sw) << 4); };
+        auto waux_bar = [&](uint32_t b) { return bar0 + 256u + 8u * (static_cast<uint32_t>(ew) * 2u + b); };
+        const bool has_bias = (EPI != kEpiMulGeluGrad) && p.bias != nullptr;
+        const ptx::f2 al = ptx::make_f2(p.alpha, p.alpha);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        uint32_t tile_i = 0;  // tiles this warp has started: bias buffer parity, position in the aux ring
+
+        // kEpiMulGeluGrad: the 32 x 64 box of the producer's pre-activation for this warp's step g
+        // (two steps per tile) lands in buffer g & 1; issued by the elected lane two steps ahead
+        auto issue_aux = [&](uint32_t g) {
+            const long long u = static_cast<long long>(first_unit) +
+                                static_cast<long long>(g >> 1) * unit_stride;
+            if (u >= num_units) return;
+            int m_blk, n_blk, split;
+            decode_unit(p, static_cast<int>(u), m_blk, n_blk, split);
+            const uint32_t ab = waux_bar(g & 1u);
+            ptx::mbar_expect_tx(ab, kBoxBytes);
+            ptx::tma_load_2d(aux0 + (g & 1u) * kBoxBytes, &tmE, ab,
+                             n_blk * BLOCK_N + hf * 128 + static_cast<int>(g & 1u) * 64,
+                             m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM + q * 32);
+        };
+        if constexpr (EPI == kEpiMulGeluGrad) {
+            if (ptx::elect_one()) {
+                issue_aux(0);
+                issue_aux(1);
+            }
+            __syncwarp();
+        }
+        auto release_acc = [&](int a) {
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(a), 0));
+                else ptx::mbar_arrive(tempty_bar(a));
+            }
+            __syncwarp();
+        };
+
+        for (int u = first_unit; u < num_units; u += unit_stride, ++tile_i) {
+            if (ptx::ld_shared_u32_volatile(epi_abort_addr) != 0) break;
+            int m_blk, n_blk, split;
+            decode_unit(p, u, m_blk, n_blk, split);
+            const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
+            const int nw = n_blk * BLOCK_N + hf * 128;  // this warp's first column
+            // this lane's four of the warp's 128 bias values, fetched while the tile is still in the
+            // tensor core
+            uint32_t bv[4] = {0u, 0u, 0u, 0u};
+            if (has_bias) {
+                const int col = nw + lane * 4;
+                if (col < p.N) {  // N is a multiple of 8 and col of 4: all four exist
+                    // element loads: the bias pointer is only required to be 2-byte aligned
+                    const unsigned short *bp = reinterpret_cast<const unsigned short *>(p.bias) + col;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) bv[k] = static_cast<uint32_t>(__ldg(bp + k)) << 16;
+                }
+            }
+            bool ok = true;
+            if (lane == 0) ok = wait_barrier(wctx, tfull_bar(acc), acc_phase, 400 + acc);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
+            ptx::tc_fence_after();
+            // The bias buffer of this parity was last read for the tile two back, whose accumulator
+            // every warp handed over (after issuing its last bias loads) before this tile's MMAs
+            // could start. The four warps of a column half write the same values.
+            const uint32_t bias_t = smem + Cfg::OFF_BIAS + (tile_i & 1u) * (BLOCK_N * 4u) +
+                                    static_cast<uint32_t>(hf) * 512u;
+            if (has_bias) {
+                ptx::st_shared_v4(bias_t + static_cast<uint32_t>(lane) * 16u, bv[0], bv[1], bv[2], bv[3]);
+                __syncwarp();
+            }
+            const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
+                                   static_cast<uint32_t>(acc * BLOCK_N + hf * 128);
+            uint32_t rr[2][32];
+            ptx::tmem_ld_32x32_issue(t_acc, rr[0]);
+            float st_m = -INFINITY, st_s = 0.0f;  // kEpiStoreStats: this thread's row statistics
+#pragma unroll
+            for (int s4 = 0; s4 < 4; ++s4) {  // 32 columns at a time; two make a stored box
+                const int step = s4 >> 1, sub = s4 & 1;
+                const uint32_t g = tile_i * 2u + static_cast<uint32_t>(step);
+                float4 bb[8];
+                if (has_bias) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        ptx::ld_shared_f32x4(bias_t + 4u * static_cast<uint32_t>(s4 * 32 + j * 4), bb[j]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) bb[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                }
+                uint32_t (&r)[32] = rr[s4 & 1];
+                ptx::tmem_ld_wait_32(r);
+                if (s4 < 3) ptx::tmem_ld_32x32_issue(t_acc + static_cast<uint32_t>((s4 + 1) * 32), rr[(s4 + 1) & 1]);
+                else release_acc(acc);  // accumulator fully read
+                if (sub == 0) {
+                    // the staging box is free once the previous step's store has read it
+                    if (ptx::elect_one()) ptx::bulk_wait_group_read<0>();
+                    __syncwarp();
+                    if (EPI == kEpiMulGeluGrad) {
+                        bool aok = true;
+                        if (lane == 0)
+                            aok = wait_barrier(wctx, waux_bar(g & 1u), (g >> 1) & 1u, 500 + ew);
+                        aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
+                        if (!aok) {
+                            ptx::st_shared_u32_volatile(epi_abort_addr, 1);
+                            ok = false;
+                        }
+                    }
+                }
+                float sv[EPI == kEpiStoreStats ? 32 : 1];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t pos = chunk_pos(sub * 4 + j);
+                    if (EPI == kEpiMulGeluGrad) {
+                        uint32_t x[4], w[4];
+                        ptx::ld_shared_v4(aux0 + (g & 1u) * kBoxBytes + pos, x[0], x[1], x[2], x[3]);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const ptx::f2 a2 = ptx::make_f2_bits(r[j * 8 + 2 * k], r[j * 8 + 2 * k + 1]);
+                            const ptx::f2 x2 = ptx::make_f2_bits(x[k] << 16, x[k] & 0xffff0000u);
+                            w[k] = pack_f2_bf16x2(mul_gelu_bwd2(a2, x2));
+                        }
+                        ptx::st_shared_v4(stg + pos, w[0], w[1], w[2], w[3]);
+                    } else {
+                        const float4 b0 = bb[2 * j], b1 = bb[2 * j + 1];
+                        ptx::f2 z[4];  // eight columns as four packed pairs
+                        z[0] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 0], r[j * 8 + 1]), al, ptx::make_f2(b0.x, b0.y));
+                        z[1] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 2], r[j * 8 + 3]), al, ptx::make_f2(b0.z, b0.w));
+                        z[2] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 4], r[j * 8 + 5]), al, ptx::make_f2(b1.x, b1.y));
+                        z[3] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 6], r[j * 8 + 7]), al, ptx::make_f2(b1.z, b1.w));
+                        if (EPI == kEpiGelu) {
+                            ptx::st_shared_v4(stg + kBoxBytes + pos, pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),
+                                              pack_f2_bf16x2(z[2]), pack_f2_bf16x2(z[3]));
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) z[k] = gelu_fwd2(z[k]);
+                        }
+                        const uint32_t w0 = pack_f2_bf16x2(z[0]), w1 = pack_f2_bf16x2(z[1]),
+                                       w2 = pack_f2_bf16x2(z[2]), w3 = pack_f2_bf16x2(z[3]);
+                        ptx::st_shared_v4(stg + pos, w0, w1, w2, w3);
+                        if (EPI == kEpiStoreStats) {  // keep the eight stored (rounded) values
+                            sv[j * 8 + 0] = ptx::bf16_lo(w0); sv[j * 8 + 1] = ptx::bf16_hi(w0);
+                            sv[j * 8 + 2] = ptx::bf16_lo(w1); sv[j * 8 + 3] = ptx::bf16_hi(w1);
+                            sv[j * 8 + 4] = ptx::bf16_lo(w2); sv[j * 8 + 5] = ptx::bf16_hi(w2);
+                            sv[j * 8 + 6] = ptx::bf16_lo(w3); sv[j * 8 + 7] = ptx::bf16_hi(w3);
+                        }
+                    }
+                }
+                if (EPI == kEpiStoreStats) {
+                    // online softmax statistics of this thread's 32 stored values: running
+                    // maximum st_m and sum of exp(value - st_m), columns >= v_real left out
+                    const int g0 = nw + s4 * 32;
+                    float mx = -INFINITY;
+                    if (g0 + 32 > p.v_real) {  // only the tile that straddles v_real masks
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            if (g0 + k >= p.v_real) sv[k] = -INFINITY;
+                    }
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, sv[k]);
+                    if (mx > st_m) {
+                        st_s *= exp2f((st_m - mx) * 1.4426950408889634f);  // 0 while st_m = -inf
+                        st_m = mx;
+                    }
+                    if (st_m > -INFINITY) {
+                        const float ms = st_m * 1.4426950408889634f;
+                        float acc_s = 0.0f;
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            acc_s += ptx::ex2_approx(fmaf(sv[k], 1.4426950408889634f, -ms));
+                        st_s += acc_s;
+                    }
+                }
+                if (sub == 1) {
+                    // the box is complete: make it visible to the TMA engine and store it
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (ptx::elect_one()) {
+                        const int x = nw + step * 64;
+                        const int y = m0 + q * 32;
+                        if (ok && x < p.N && y < p.M) {
+                            ptx::tma_store_2d(&tmD, stg, x, y);
+                            if (EPI == kEpiGelu) ptx::tma_store_2d(&tmE, stg + kBoxBytes, x, y);
+                        }
+                        ptx::bulk_commit_group();
+                        // every lane has read this step's pre-activation box (__syncwarp above)
+                        if (EPI == kEpiMulGeluGrad) issue_aux(g + 2u);
+                    }
+                    __syncwarp();
+                }
+            }
+            if (EPI == kEpiStoreStats) {
+                const long long grow = static_cast<long long>(m0) + row;
+                if (ok && grow < p.M)
+                    p.stats[grow * p.stats_ld + n_blk * 2 + hf] = make_float2(st_m, st_s);
+            }
+            if (++acc == 2) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
+        }
+        if (ptx::elect_one()) ptx::bulk_wait_group<0>();  // all stores have reached global memory
+        __syncwarp();
+      } else {
         // TMA stores and the bulk-group bookkeeping are issued by one elected lane of warp 2, always
         // from a warp-uniform branch with the election at the point of use
         const bool store_warp = (warp == 2);
@@ -798,6 +1028,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (store_warp) {
             if (ptx::elect_one()) ptx::bulk_wait_group<0>();  // all stores have reached global memory
         }
+      }
     }
 
     // ---------------------------------------------------------------- common exit

@@ -227,9 +227,9 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     // operands are fetched as 64 x 64 boxes; results (and the aux tile) move as 128-row chunks
     if ((rc = get_tmap(s, &tA, a.A, a.a_rows, a.a_cols, 0, 64)) != NB_OK) return rc;
     if ((rc = get_tmap(s, &tB, a.B, a.b_rows, a.b_cols, 0, 64)) != NB_OK) return rc;
-    if ((rc = get_tmap(s, &tD, a.D, a.d_rows, a.d_cols, a.d_dtype, kBlockM)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tD, a.D, a.d_rows, a.d_cols, a.d_dtype, Cfg::OUT_BOX_ROWS)) != NB_OK) return rc;
     if (a.E) {
-        if ((rc = get_tmap(s, &tE, a.E, a.e_rows, a.e_cols, 0, kBlockM)) != NB_OK) return rc;
+        if ((rc = get_tmap(s, &tE, a.E, a.e_rows, a.e_cols, 0, Cfg::OUT_BOX_ROWS)) != NB_OK) return rc;
     } else {
         tE = tD;
     }

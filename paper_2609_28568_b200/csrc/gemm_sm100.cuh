@@ -99,9 +99,11 @@ struct GemmCfg {
     // Warp-private epilogue (bf16 results of full-width tiles): every epilogue warp stages and
     // stores its own 32-row boxes, no barrier joins the warps. The bias then lives in two buffers
     // (by tile parity) and each warp has its own pair of pre-activation barriers.
-    static constexpr bool WARP_EPI = BLOCK_N_ == 256 && !DBIAS_ &&
+    static constexpr bool WARP_EPI = BLOCK_N_ == 256 &&
                                      (EPI_ == kEpiStore || EPI_ == kEpiStoreStats || EPI_ == kEpiGelu ||
-                                      EPI_ == kEpiMulGeluGrad);
+                                      EPI_ == kEpiMulGeluGrad || EPI_ == kEpiF32);
+    // boxes of staging per epilogue warp: one per stored plane; fp32 results alternate between two
+    static constexpr int WARP_BOXES = (EPI_ == kEpiF32) ? 2 : (EPI_ == kEpiGelu) ? 2 : 1;
     static constexpr int OUT_BOX_ROWS = WARP_EPI ? 32 : kBlockM;
     static constexpr uint32_t BIAS_BYTES = (WARP_EPI ? 2 : 1) * BLOCK_N * 4;
     static constexpr uint32_t OFF_BAR = OFF_BIAS + BIAS_BYTES;
@@ -123,7 +125,7 @@ struct GemmCfg {
     static_assert(EPI != kEpiMulGeluGrad || SLOTS >= 2, "staging ring");
     static_assert(EPI != kEpiSwiglu || BLOCK_N == 256, "SwiGLU tiles pair 128 gate + 128 up cols");
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
-    static_assert(!WARP_EPI || NSTG * kStgBytes >= 8u * BUFS_PER_STEP * 4096u, "a box per warp and plane");
+    static_assert(!WARP_EPI || NSTG * kStgBytes >= 8u * WARP_BOXES * 4096u, "staging boxes per warp");
     static_assert(!WARP_EPI || EPI_ != kEpiMulGeluGrad || NAUX * kStgBytes >= 8u * 2u * 4096u,
                   "two pre-activation boxes per warp");
     static_assert(!DBIAS_ || (A_MN_ && EPI_ == kEpiF32), "the fused bias gradient belongs to wgrad");
@@ -547,14 +549,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // TMEM, a proxy fence or a store, the others compute.
         const int ew = warp - 2;                  // 0..7
         constexpr uint32_t kBoxBytes = 32 * 128;  // 32 rows x 64 bf16, 128-byte swizzled
-        constexpr uint32_t NBUF = Cfg::BUFS_PER_STEP;  // 1; kEpiGelu: activated + pre-activation
+        constexpr uint32_t NBUF = Cfg::WARP_BOXES;  // kEpiGelu: activated + pre-activation; kEpiF32: a ring of two
         const uint32_t stg = smem + Cfg::OFF_STG + static_cast<uint32_t>(ew) * NBUF * kBoxBytes;
         const uint32_t aux0 = smem + Cfg::OFF_AUX + static_cast<uint32_t>(ew) * 2u * kBoxBytes;
         const uint32_t lane_off = static_cast<uint32_t>(lane) * 128u;
         const uint32_t sw = static_cast<uint32_t>(lane & 7);
         auto chunk_pos = [&](int chunk) { return lane_off + ((static_cast<uint32_t>(chunk) ^ sw) << 4); };
         auto waux_bar = [&](uint32_t b) { return bar0 + 256u + 8u * (static_cast<uint32_t>(ew) * 2u + b); };
-        const bool has_bias = (EPI != kEpiMulGeluGrad) && p.bias != nullptr;
+        const bool has_bias = (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiGelu) && p.bias != nullptr;
         const ptx::f2 al = ptx::make_f2(p.alpha, p.alpha);
         int acc = 0;
         uint32_t acc_phase = 0;
@@ -625,26 +627,78 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                    static_cast<uint32_t>(acc * BLOCK_N + hf * 128);
-            uint32_t rr[2][32];
-            ptx::tmem_ld_32x32_issue(t_acc, rr[0]);
+            // All four loads of the warp's 128 columns are issued at once (a TMEM load takes several
+            // hundred cycles while the tensor core is busy; one after the other they would add up),
+            // unless the register budget of the kernel only allows two in flight.
+            constexpr int LD_DEPTH = Cfg::DBIAS ? 2 : 4;
+            uint32_t rr[LD_DEPTH][32];
+#pragma unroll
+            for (int i = 0; i < LD_DEPTH; ++i)
+                ptx::tmem_ld_32x32_issue(t_acc + static_cast<uint32_t>(i * 32), rr[i]);
             float st_m = -INFINITY, st_s = 0.0f;  // kEpiStoreStats: this thread's row statistics
 #pragma unroll
             for (int s4 = 0; s4 < 4; ++s4) {  // 32 columns at a time; two make a stored box
                 const int step = s4 >> 1, sub = s4 & 1;
                 const uint32_t g = tile_i * 2u + static_cast<uint32_t>(step);
-                float4 bb[8];
-                if (has_bias) {
+                // the bias of 16 columns at a time, ahead of the arithmetic that uses it (the loads
+                // cannot be moved by the compiler across the shared-memory stores in between)
+                float4 bb[4];
+                auto load_bias16 = [&](int half) {
+                    if (has_bias) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            ptx::ld_shared_f32x4(bias_t + 4u * static_cast<uint32_t>(s4 * 32 + half * 16 + j * 4),
+                                                 bb[j]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) bb[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    }
+                };
+                load_bias16(0);
+                uint32_t (&r)[32] = rr[s4 % LD_DEPTH];
+                if (LD_DEPTH == 4) {
+                    if (s4 == 0) {  // one wait covers all four loads
+                        ptx::tmem_ld_wait_32(rr[0]);
+                        ptx::reg_fence_32(rr[1 % LD_DEPTH]);
+                        ptx::reg_fence_32(rr[2 % LD_DEPTH]);
+                        ptx::reg_fence_32(rr[3 % LD_DEPTH]);
+                    }
+                } else {
+                    // waits for every load issued so far: the one in use and the one after it
+                    ptx::tmem_ld_wait_32(r);
+                    ptx::reg_fence_32(rr[(s4 + 1) % LD_DEPTH]);
+                }
+                // The accumulator goes back once its last column is in registers. Where there is a
+                // bias, the hand-over also orders the reuse of the bias buffers, so it waits until
+                // this tile's last bias loads have been issued (in the loop over j below).
+                constexpr bool kBiasEpi = (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiGelu);
+                constexpr int kReleaseAt = (LD_DEPTH == 4) ? 0 : 3;
+                if (!kBiasEpi && s4 == kReleaseAt) release_acc(acc);
+                if constexpr (EPI == kEpiF32) {
+                    // 32 fp32 columns are a box of their own; two boxes alternate, so a box is
+                    // rewritten only after the copy issued two boxes ago has read it
+                    const uint32_t fb = stg + static_cast<uint32_t>(s4 & 1) * kBoxBytes;
+                    if (ptx::elect_one()) ptx::bulk_wait_group_read<1>();
+                    __syncwarp();
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        ptx::ld_shared_f32x4(bias_t + 4u * static_cast<uint32_t>(s4 * 32 + j * 4), bb[j]);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) bb[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                        ptx::st_shared_v4(fb + chunk_pos(j), r[j * 4], r[j * 4 + 1], r[j * 4 + 2], r[j * 4 + 3]);
+                    if (LD_DEPTH == 2 && s4 + 2 < 4)  // these registers are free again
+                        ptx::tmem_ld_32x32_issue(t_acc + static_cast<uint32_t>((s4 + 2) * 32), rr[s4 % LD_DEPTH]);
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (ptx::elect_one()) {
+                        const int x = nw + s4 * 32;
+                        const int y = m0 + q * 32;
+                        if (ok && x < p.N && y < p.M) {
+                            if (p.reduce) ptx::tma_reduce_add_2d(&tmD, fb, x, y);
+                            else ptx::tma_store_2d(&tmD, fb, x, y);
+                        }
+                        ptx::bulk_commit_group();
+                    }
+                    __syncwarp();
+                    continue;
                 }
-                uint32_t (&r)[32] = rr[s4 & 1];
-                ptx::tmem_ld_wait_32(r);
-                if (s4 < 3) ptx::tmem_ld_32x32_issue(t_acc + static_cast<uint32_t>((s4 + 1) * 32), rr[(s4 + 1) & 1]);
-                else release_acc(acc);  // accumulator fully read
                 if (sub == 0) {
                     // the staging box is free once the previous step's store has read it
                     if (ptx::elect_one()) ptx::bulk_wait_group_read<0>();
@@ -675,7 +729,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         }
                         ptx::st_shared_v4(stg + pos, w[0], w[1], w[2], w[3]);
                     } else {
-                        const float4 b0 = bb[2 * j], b1 = bb[2 * j + 1];
+                        if (j == 2) {
+                            load_bias16(1);
+                            if (s4 == 3) release_acc(acc);  // kBiasEpi: the tile's last bias loads are out
+                        }
+                        const float4 b0 = bb[2 * (j & 1)], b1 = bb[2 * (j & 1) + 1];
                         ptx::f2 z[4];  // eight columns as four packed pairs
                         z[0] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 0], r[j * 8 + 1]), al, ptx::make_f2(b0.x, b0.y));
                         z[1] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 2], r[j * 8 + 3]), al, ptx::make_f2(b0.z, b0.w));

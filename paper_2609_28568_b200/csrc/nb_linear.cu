@@ -300,7 +300,7 @@ using FwdGelu1 = GemmCfg<1, 256, 3, 4, false, false, kEpiGelu>;
 using FwdSwiglu1 = GemmCfg<1, 256, 3, 3, false, false, kEpiSwiglu>;
 using DgradStore1 = GemmCfg<1, 256, 4, 2, false, true, kEpiStore>;
 using DgradMulGelu1 = GemmCfg<1, 256, 2, 2, false, true, kEpiMulGeluGrad>;
-using WgradF32_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32>;
+using WgradF32_1 = GemmCfg<1, 256, 3, 4, true, true, kEpiF32>;
 using WgradBf16_1 = GemmCfg<1, 256, 4, 2, true, true, kEpiStore>;
 using FwdStore2 = GemmCfg<2, 256, 6, 2, false, false, kEpiStore>;
 using FwdStoreStats1 = GemmCfg<1, 256, 4, 2, false, false, kEpiStoreStats>;
@@ -309,9 +309,9 @@ using FwdGelu2 = GemmCfg<2, 256, 5, 4, false, false, kEpiGelu>;
 using FwdSwiglu2 = GemmCfg<2, 256, 5, 3, false, false, kEpiSwiglu>;
 using DgradStore2 = GemmCfg<2, 256, 6, 2, false, true, kEpiStore>;
 using DgradMulGelu2 = GemmCfg<2, 256, 4, 2, false, true, kEpiMulGeluGrad>;
-using WgradF32_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32>;
-using WgradF32Bias1 = GemmCfg<1, 256, 4, 2, true, true, kEpiF32, true>;
-using WgradF32Bias2 = GemmCfg<2, 256, 6, 2, true, true, kEpiF32, true>;
+using WgradF32_2 = GemmCfg<2, 256, 5, 4, true, true, kEpiF32>;
+using WgradF32Bias1 = GemmCfg<1, 256, 3, 4, true, true, kEpiF32, true>;
+using WgradF32Bias2 = GemmCfg<2, 256, 5, 4, true, true, kEpiF32, true>;
 using WgradBf16_2 = GemmCfg<2, 256, 6, 2, true, true, kEpiStore>;
 // Narrow results (N <= 64: the rank-r products of the adapter layer). A 256-wide tile would spend
 // 4-16x the tensor-core time on padding; a 64-wide one leaves these products bound by the read of

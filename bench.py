@@ -192,7 +192,13 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from the host in the timed region instead of replaying a CUDA graph")
+    ap.add_argument("--dp", action="store_true",
+                    help="data parallel instead of replicas: the same weights on every rank, its own rows, and "
+                         "the fp32 gradients all-reduced (NCCL) in buckets under the last micro-step's backward; "
+                         "launches eagerly (no graph)")
     args = ap.parse_args()
+    if args.dp:
+        args.no_graph = True
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 
@@ -220,7 +226,15 @@ def main():
 
     model, BT, micro_steps, cfg_id, wgrad, wdesc = WORKLOADS[args.workload]
     stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
-                        wgrad=wgrad)
+                        wgrad=wgrad, shared_weights=args.dp)
+    reducer = None
+    if args.dp:
+        from paper_2609_28568_b200 import dp as dpmod
+        if not wgrad:
+            raise SystemExit("--dp needs a workload with weight gradients")
+        fp = torch.stack([t.float().sum() for t in stack.input_tensors(0)])
+        dpmod.assert_ranks_differ(fp, dist, "inputs")
+        reducer = dpmod.GradAllReducer(stack.attach_gradient_buckets(), dist, average=True)
     # reserve the activation-backward workspace before timing so no call allocates
     need = max((BT * L.spec.OC * 2 for L in stack.layers
                 if L.spec.act != shapes.ACT_NONE and L.dz_from is None), default=0)
@@ -237,7 +251,10 @@ def main():
 
     # ---- warm-up
     for _ in range(args.warmup):
-        stack.step()
+        if reducer is not None:
+            stack.step_dp(reducer)
+        else:
+            stack.step()
     nb.nb_check_status()
 
     # ---- timed region: K steps between two events on the launch stream. No events between the
@@ -260,6 +277,8 @@ def main():
     # capturable: no allocation, no synchronisation) and the timed region replays it, so the
     # 588 launches of a step cost the host one call.
     run_step, launches_per_step = stack.step, None
+    if reducer is not None:
+        run_step = lambda: stack.step_dp(reducer)  # noqa: E731
     if not args.no_graph:
         cap = torch.cuda.Stream(device=dev)
         cap.wait_stream(torch.cuda.current_stream())
@@ -364,7 +383,9 @@ def main():
             "config": {"workload": args.workload, "description": wdesc, "BT": BT,
                        "micro_steps": micro_steps, "l2": "inputs_exceed_l2 (a step touches >20 GB)",
                        "launch": "eager" if args.no_graph else "cuda_graph_replay",
-                       "parallelism": f"replicas x{world}, no collective"},
+                       "parallelism": (f"dp{world}: fp32 gradient all-reduce in {len(reducer.b.buckets)} buckets "
+                                       f"under the last micro-step's backward" if reducer is not None
+                                       else f"replicas x{world}, no collective")},
             "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches),
         }

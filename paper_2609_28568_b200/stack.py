@@ -39,7 +39,8 @@ class _Layer:
 
 class LinearStack:
     def __init__(self, model: str, BT: int, micro_steps: int, device="cuda", config_id: int = 4,
-                 seed_offset: int = 0, wgrad: bool = True, generate: bool = True):
+                 seed_offset: int = 0, wgrad: bool = True, generate: bool = True,
+                 shared_weights: bool = False):
         self.model, self.BT, self.micro_steps, self.device = model, BT, micro_steps, device
         self.wgrad = wgrad
         self.layers: list[_Layer] = []
@@ -67,6 +68,9 @@ class LinearStack:
         if head is not None:
             self.layers.append(_Layer(head, idx))
         self.config_id, self.seed_offset = config_id, seed_offset
+        # data parallel: every rank holds the same weights and its own rows (seed_offset = rank
+        # then only moves the activations and output gradients); replicas differ in everything
+        self.shared_weights = shared_weights
         self._allocate()
         if generate:
             self.generate_inputs()
@@ -90,7 +94,8 @@ class LinearStack:
                 L.dout.append(None if L.dz_from else torch.empty((BT, s.out_cols), dtype=bf, device=dev))
 
     def seed(self, L: _Layer, role: int, ms: int = 0) -> int:
-        return synth.tensor_seed(self.config_id, L.index, role, ms) + 100000 * self.seed_offset
+        off = 0 if (self.shared_weights and role in (1, 2)) else self.seed_offset
+        return synth.tensor_seed(self.config_id, L.index, role, ms) + 100000 * off
 
     def generate_inputs(self):
         """Fill weights, biases and per-micro-step inputs / output gradients from their seeds."""
@@ -178,3 +183,43 @@ class LinearStack:
         """One pass of the whole path: every micro-step, forward then backward."""
         for ms in range(self.micro_steps):
             self.micro_step(ms, hook)
+
+    # ------------------------------------------------------------------ data parallel
+    def attach_gradient_buckets(self, bucket_bytes: int = 32 << 20):
+        """Move the fp32 gradients into one flat buffer, in the order backward finalises them
+        (last layer first; weight, then bias), cut into buckets for the all-reduce. Returns the
+        `GradientBuckets`; the layers' `dweight` / `dbias` become views of it."""
+        from .dp import GradientBuckets
+        if not self.wgrad:
+            raise ValueError("this stack computes no weight gradients")
+        entries = []
+        for L in reversed(self.layers):
+            entries.append((("dweight", L.index), tuple(L.dweight.shape)))
+            if L.dbias is not None:
+                entries.append((("dbias", L.index), tuple(L.dbias.shape)))
+        gb = GradientBuckets(entries, bucket_bytes, self.device)
+        for L in self.layers:
+            L.dweight = gb.view(("dweight", L.index))
+            if L.dbias is not None:
+                L.dbias = gb.view(("dbias", L.index))
+        return gb
+
+    def step_dp(self, reducer, hook=None):
+        """`step()` with the gradient exchange: during the LAST micro-step's backward every layer's
+        gradients are reported final as soon as its backward call is enqueued, so a bucket's
+        all-reduce runs under the backward of the layers below it; returns after `finish()`."""
+        reducer.begin_step()
+        last = self.micro_steps - 1
+
+        def on_call(kind, L, begin):
+            if hook:
+                hook(kind, L, begin)
+            if kind == "bwd" and not begin:
+                reducer.mark_ready(("dweight", L.index))
+                if L.dbias is not None:
+                    reducer.mark_ready(("dbias", L.index))
+
+        for ms in range(self.micro_steps):
+            self.forward(ms, hook)
+            self.backward(ms, on_call if ms == last else hook)
+        reducer.finish()

@@ -169,6 +169,84 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_library(args, rank, local_rank):
+    """Context, not a contract arm: the same stack composed from the framework's library ops
+    (cuBLAS GEMMs, separate bias / GELU / GELU-backward / reduction / accumulation kernels) on one
+    GPU, and its bare GEMMs alone. None of this repository's kernels run here."""
+    if rank != 0:
+        return
+    import torch
+    import torch.nn.functional as F
+    from paper_2609_28568_b200 import shapes
+    from paper_2609_28568_b200.stack import LinearStack
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    model, BT, micro_steps, cfg_id, wgrad, wdesc = WORKLOADS[args.workload]
+    stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, wgrad=wgrad)
+    if any(L.spec.act == shapes.ACT_SWIGLU for L in stack.layers):
+        raise SystemExit("--impl library covers the GPT-2 workloads only")
+
+    def step(full: bool):
+        for ms in range(micro_steps):
+            for L in stack.layers:
+                x = stack.layer_inp(L, ms)
+                if not full:
+                    F.linear(x, L.weight)
+                    continue
+                y = F.linear(x, L.weight, L.bias)
+                if L.spec.act == shapes.ACT_GELU:
+                    L.pre, y = y, F.gelu(y, approximate="tanh")
+                L.out = y
+            for L in reversed(stack.layers):
+                dz = L.dz_from.dinp if L.dz_from is not None else L.dout[ms]
+                x = stack.layer_inp(L, ms)
+                if not full:
+                    dz @ L.weight
+                    if wgrad:
+                        dz.t() @ x
+                    continue
+                dx = dz @ L.weight
+                if L.chained_from is not None:  # the producer's GELU backward as its own kernel
+                    dx = torch.ops.aten.gelu_backward(dx, L.chained_from.pre, approximate="tanh")
+                L.dinp = dx
+                if wgrad:
+                    g = dz.t() @ x              # bf16 product, then the fp32 accumulation
+                    if ms == 0:
+                        L.dweight.copy_(g)
+                    else:
+                        L.dweight.add_(g)
+                    if L.dbias is not None:
+                        b = dz.sum(0, dtype=torch.float32)
+                        if ms == 0:
+                            L.dbias.copy_(b)
+                        else:
+                            L.dbias.add_(b)
+
+    flops = stack.flops_per_micro_step() * micro_steps
+    res = {}
+    for name, full in (("composed", True), ("gemms_only", False)):
+        for _ in range(max(args.warmup, 2)):
+            step(full)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step(full)
+        e1.record()
+        torch.cuda.synchronize()
+        ms_step = e0.elapsed_time(e1) / args.steps
+        res[name] = {"ms_per_step": ms_step, "tflops": flops / (ms_step * 1e-3) / 1e12}
+    print(json.dumps({
+        "impl": "library", "metric": "gpt2_124m_linear_fwd_bwd_tflops", "value": res["composed"]["tflops"],
+        "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": res["composed"]["ms_per_step"], "higher_is_better": True, "dtype": "bf16",
+        "data": "synthetic", "config": {"workload": args.workload, "description": wdesc},
+        "gemms_only": res["gemms_only"],
+        "note": "framework library ops (cuBLAS GEMMs + separate elementwise / reduction kernels); "
+                "gemms_only = the bare bf16 GEMMs without bias, GELU, gradient accumulation",
+    }), flush=True)
+
+
 def max_over_ranks(value: float, dist, device) -> float:
     """The slowest rank's figure (a job is as slow as its slowest replica)."""
     if dist is None:
@@ -185,7 +263,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "library"],
+                    help="ours; reference = the CPU oracle (the contract's reference arm); library = the same "
+                         "stack from cuBLAS and framework kernels, for context")
     ap.add_argument("--workload", default="gpt2_124m_stack", choices=sorted(WORKLOADS))
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -208,6 +288,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.impl == "library":
+        run_library(args, rank, local_rank)
         return
 
     import torch

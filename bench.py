@@ -346,11 +346,19 @@ def main():
     records = []  # (kind, layer name, start event, end event), filled by the breakdown pass
 
     def hook(kind, L, begin):
+        # one event per call boundary: a call's end is the next call's start (the calls of a step
+        # follow one another without gaps), which halves the events the breakdown pass inserts
+        if begin:
+            e = torch.cuda.Event(enable_timing=True)
+            e.record()
+            if records and records[-1][3] is None:
+                records[-1][3] = e
+            records.append([kind, L.spec.name, e, None])
+
+    def close_records():
         e = torch.cuda.Event(enable_timing=True)
         e.record()
-        if begin:
-            records.append([kind, L.spec.name, e, None])
-        else:
+        if records and records[-1][3] is None:
             records[-1][3] = e
 
     props = torch.cuda.get_device_properties(dev)
@@ -396,6 +404,7 @@ def main():
     bev0.record()
     for _ in range(args.steps):
         stack.step(hook)
+    close_records()
     bev1.record()
     barrier()
     clocks = sampler.stop()
@@ -423,7 +432,14 @@ def main():
     # that is the "kernel timed inside a long step" case, compared with the sustained peak
     long_step = ms_per_step * (args.warmup + 2 * args.steps) > 1000.0
     peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
-    achieved_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    # Every launch of a step is an instantiation of the one GEMM kernel, so its average launch
+    # duration over the timed region is that region's length / launches, and algorithmic flops per
+    # launch / that duration is this rank's flops / time of the timed region. (The breakdown pass
+    # below it has events between the calls, which cost it dependent-launch overlap: it is only
+    # used for the per-call split.)
+    my_ms_per_step = ev0.elapsed_time(ev1) / args.steps
+    achieved_tf = flops_step / (my_ms_per_step * 1e-3) / 1e12
+    breakdown_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
@@ -435,9 +451,14 @@ def main():
         "bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
         "frac": achieved_tf / peak_tf, "traffic": traffic,
         "peak_source": f"{peak_src} cuBLAS bf16 ({'sustained' if long_step else 'burst'})",
-        "kernel": "nb::gemm_kernel (tcgen05 fwd / dgrad / wgrad instantiations), all launches of a step; "
-                  "durations from a second pass over the same steps with events around every call",
+        "kernel": "nb::gemm_kernel (tcgen05 fwd / dgrad / wgrad instantiations): every launch of a step; "
+                  "average launch duration = timed region (CUDA events on the launch stream) / launches; "
+                  "per_call from a second pass over the same steps with an event at every call boundary",
+        "launches_per_step": launches / args.steps,
+        "avg_launch_us": my_ms_per_step * 1e3 / (launches / args.steps) if launches else None,
+        "flops_per_launch": flops_step / (launches / args.steps) if launches else None,
         "breakdown_pass_ms_per_step": breakdown_ms_per_step,
+        "breakdown_pass_tflops": breakdown_tf,
         "frac_of_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
         "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
         "frac_of_sustained_peak": achieved_tf / peaks["bf16_tflops_sustained"],

@@ -678,7 +678,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     // 32 fp32 columns are a box of their own; two boxes alternate, so a box is
                     // rewritten only after the copy issued two boxes ago has read it
                     const uint32_t fb = stg + static_cast<uint32_t>(s4 & 1) * kBoxBytes;
-                    if (ptx::elect_one()) ptx::bulk_wait_group_read<1>();
+                    ptx::bulk_wait_group_read<1>();  // every lane: only the one that issued copies has any to wait for
                     __syncwarp();
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
@@ -701,7 +701,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
                 if (sub == 0) {
                     // the staging box is free once the previous step's store has read it
-                    if (ptx::elect_one()) ptx::bulk_wait_group_read<0>();
+                    ptx::bulk_wait_group_read<0>();  // every lane: only the one that issued copies has any to wait for
                     __syncwarp();
                     if (EPI == kEpiMulGeluGrad) {
                         bool aok = true;
@@ -809,7 +809,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 acc_phase ^= 1u;
             }
         }
-        if (ptx::elect_one()) ptx::bulk_wait_group<0>();  // all stores have reached global memory
+        ptx::bulk_wait_group<0>();  // all stores have reached global memory (every lane waits for its own)
         __syncwarp();
       } else {
         // TMA stores and the bulk-group bookkeeping are issued by one elected lane of warp 2, always

@@ -545,3 +545,28 @@ def test_flat_gradient_buckets_give_the_same_gradients_on_one_rank():
         assert Lb.dweight.data_ptr() % 16 == 0
         assert rel_frob(f32(Lb.dweight), f32(La.dweight)) < 1e-5
         assert rel_frob(f32(Lb.dbias), f32(La.dbias)) < 1e-5
+
+
+@pytest.mark.parametrize("act", [nb.ACT_NONE, nb.ACT_GELU])
+def test_bias_reaches_every_tile_full_tensor(act):
+    """Every element of a many-tile result carries ITS column's bias: the result with a large bias
+    equals the bias-free result plus the bias, to the rounding of the two bf16 conversions. (The
+    epilogue warps keep the bias in buffers they reuse from tile to tile without a barrier.)"""
+    BT, C, OC = 16384, 768, 3072 if act == nb.ACT_GELU else 2304
+    inp = gen(7001, (BT, C), 1.0)
+    w = gen(7002, (OC, C), 0.02)
+    b = gen(7003, (OC,), 1.0)
+    out_b = torch.empty((BT, OC), dtype=torch.bfloat16, device=DEV)
+    pre_b = torch.empty((BT, OC), dtype=torch.bfloat16, device=DEV) if act != nb.ACT_NONE else None
+    out_0 = torch.empty_like(out_b)
+    pre_0 = torch.empty_like(out_b) if act != nb.ACT_NONE else None
+    for _ in range(3):  # repeated launches: persistent CTAs walk different tile sequences
+        nb.nb_linear_forward_ex(out_b, pre_b, inp, w, b, BT, C, OC, act)
+    nb.nb_linear_forward_ex(out_0, pre_0, inp, w, None, BT, C, OC, act)
+    got = (pre_b if act != nb.ACT_NONE else out_b).float()
+    base = (pre_0 if act != nb.ACT_NONE else out_0).float()
+    expect = base + b.float()[None, :]
+    err = (got - expect).abs()
+    bound = 2.0 ** -7 * expect.abs() + 2.0 ** -8 * base.abs() + 1e-3
+    bad = err > bound
+    assert not bool(bad.any()), f"{int(bad.sum())} elements carry a wrong bias, worst {float(err.max()):.3f}"

@@ -570,3 +570,42 @@ def test_bias_reaches_every_tile_full_tensor(act):
     bound = 2.0 ** -7 * expect.abs() + 2.0 ** -8 * base.abs() + 1e-3
     bad = err > bound
     assert not bool(bad.any()), f"{int(bad.sum())} elements carry a wrong bias, worst {float(err.max()):.3f}"
+
+
+def test_results_beyond_two_to_the_31_elements():
+    """The largest case: 49152 rows on the padded vocabulary, 2.47e9 logits (> 2^31 elements, 4.9 GB).
+    Rows from the far end of every tensor are checked against the oracle: head forward with the
+    statistics, the in-place gradient of the loss, and the head's backward products."""
+    BT, C, Vp, V = 49152, 768, shapes.VOCAB_PADDED, shapes.VOCAB_REAL
+    assert BT * Vp > 2 ** 31
+    inp = gen(7100, (BT, C), 1.0)
+    w = gen(7101, (Vp, C), 0.02)
+    w[V:].zero_()
+    g = torch.Generator().manual_seed(7102)
+    targets = torch.randint(0, V, (BT,), generator=g, dtype=torch.int32).to(DEV)
+    logits = torch.empty((BT, Vp), dtype=torch.bfloat16, device=DEV)
+    loss = torch.empty((BT,), dtype=torch.float32, device=DEV)
+    lse = torch.empty((BT,), dtype=torch.float32, device=DEV)
+    nb.nb_lm_head_ce_forward(logits, loss, lse, inp, w, targets, BT, C, Vp, V)
+    rows = np.concatenate([sample_indices(BT, 16, 7103), np.arange(BT - 8, BT)])
+    rows = np.unique(rows)
+    rt = torch.as_tensor(rows, device=DEV)
+    o_ref, _ = oracle.linear_forward(f32(inp[rt]), f32(w))
+    check_bf16(logits[rt], o_ref, "logits rows")
+    gscale = 1.0 / BT
+    l_ref, lse_ref, d_ref = oracle.cross_entropy(f32(logits[rt]), targets[rt].cpu().numpy(), V, gscale)
+    assert np.max(np.abs(f32(loss[rt]) - l_ref)) < 1e-3
+    assert bool(torch.isfinite(loss).all())
+    nb.nb_ce_backward(logits, logits, lse, targets, gscale, BT, Vp, V)  # in place: logits become dlogits
+    dl = logits
+    check_bf16(dl[rt], d_ref, "dlogits rows")
+    assert torch.all(dl[BT - 64:, V:] == 0)
+    dinp, dw, _ = nb.linear_backward(dl, inp, w, need_dbias=False)
+    r = oracle.linear_backward(f32(dl[rt]), None, f32(w), want=("dinp",))
+    check_bf16(dinp[rt], r["dinp"], "dinp rows")
+    # weight-gradient rows (sums over all 49152 rows): a few vocabulary rows, every column
+    orow = sample_indices(V, 6, 7104)
+    ot = torch.as_tensor(orow, device=DEV)
+    rw = oracle.linear_backward(f32(dl[:, ot]), f32(inp), f32(w[ot]), want=("dweight",))
+    check_f32(dw[ot], rw["dweight"], "dweight rows")
+    assert torch.all(dw[V:] == 0)

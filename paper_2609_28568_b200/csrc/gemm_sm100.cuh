@@ -136,7 +136,7 @@ struct GemmCfg {
 //   [S, 2S)     empty[s]    MMA -> TMA
 //   2S, 2S+1    tmem_full   MMA -> epilogue
 //   2S+2, 2S+3  tmem_empty  epilogue -> MMA
-//   2S+4 .. +7  aux_full    TMA -> epilogue (kEpiMulGeluGrad), one per buffer of the aux ring
+//   byte 256 + 8 (2 w + b): kEpiMulGeluGrad, pre-activation box b (0 / 1) of epilogue warp w has landed
 //   byte 240: TMEM base address, 244: abort flag (any role), 248: epilogue abort flag
 
 struct WaitCtx {
@@ -294,7 +294,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
     auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
-    auto aux_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 4 + b); };
     // DBIAS only: a stage is handed MMA -> reducers (empty_bar) -> producer (free_bar)
     auto free_bar = [&](int s) { return bar0 + 8u * (2 * STAGES + 8 + s); };
     const uint32_t tmem_slot = bar0 + 240;
@@ -312,7 +311,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ptx::mbar_init(tfull_bar(b), 1);
             ptx::mbar_init(tempty_bar(b), kEpiWarps * CG);  // one arrive per epilogue warp of the tile
         }
-        for (int b = 0; b < 4; ++b) ptx::mbar_init(aux_bar(b), 1);
         if (Cfg::WARP_EPI && EPI == kEpiMulGeluGrad)  // two per epilogue warp, above the common slots
             for (int b = 0; b < 2 * kEpiWarps; ++b) ptx::mbar_init(bar0 + 256u + 8u * b, 1);
         ptx::st_shared_u32_volatile(abort_addr, 0);
@@ -812,8 +810,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         ptx::bulk_wait_group<0>();  // all stores have reached global memory (every lane waits for its own)
         __syncwarp();
       } else {
+        // ------------------------------------------------------------ epilogue, eight warps in step
+        // The form the 64-wide narrow tiles (plain store, fp32) and the SwiGLU epilogue use: two
+        // warps share each lane quarter and split every step's columns in halves (hf = 0 / 1); a
+        // named barrier joins the eight warps at every step and warp 2 stores the 128-row chunk.
         // TMA stores and the bulk-group bookkeeping are issued by one elected lane of warp 2, always
         // from a warp-uniform branch with the election at the point of use
+        static_assert(EPI == kEpiStore || EPI == kEpiSwiglu || EPI == kEpiF32,
+                      "the other epilogues exist only in the warp-by-warp form");
         const bool store_warp = (warp == 2);
         const int et = static_cast<int>(threadIdx.x) - 64;  // 0..255
         const uint32_t stg0 = smem + Cfg::OFF_STG;
@@ -825,33 +829,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint32_t gstep = 0;  // epilogue steps done so far (drives the staging ring)
         constexpr int SLOTS = Cfg::SLOTS;
         constexpr int STEPS = Cfg::STEPS;
-        constexpr int AUX_AHEAD = Cfg::NAUX;  // steps the pre-activation prefetch runs ahead
-
-        // coordinates of the aux tile for global step g (kEpiMulGeluGrad)
-        auto issue_aux = [&](uint32_t g) {
-            const int ui = static_cast<int>(g / STEPS);
-            const int c = static_cast<int>(g % STEPS);
-            const long long u = static_cast<long long>(first_unit) +
-                                static_cast<long long>(ui) * unit_stride;
-            if (u >= num_units) return;
-            int m_blk, n_blk, split;
-            decode_unit(p, static_cast<int>(u), m_blk, n_blk, split);
-            const int x = n_blk * BLOCK_N + c * 64;
-            const uint32_t slot = g % (Cfg::NAUX > 0 ? Cfg::NAUX : 1);
-            const uint32_t ab = aux_bar(static_cast<int>(slot));
-            ptx::mbar_expect_tx(ab, kStgBytes);
-            ptx::tma_load_2d(smem + Cfg::OFF_AUX + slot * kStgBytes, &tmE, ab, x,
-                             m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM);
-        };
-        if constexpr (EPI == kEpiMulGeluGrad) {
-            if (store_warp) {
-                if (ptx::elect_one()) {
-                    for (int g = 0; g < AUX_AHEAD; ++g) issue_aux(static_cast<uint32_t>(g));
-                }
-            }
-        }
-        __syncwarp();
-
         // the accumulator is handed back on the leader CTA's barrier
         auto release_acc = [&](int a) {
             ptx::tc_fence_before();
@@ -873,7 +850,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             decode_unit(p, u, m_blk, n_blk, split);
             const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
             const int n0 = (EPI == kEpiSwiglu) ? n_blk * 128 : n_blk * BLOCK_N;
-            if (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiGelu || EPI == kEpiSwiglu) {
+            if (EPI == kEpiStore || EPI == kEpiSwiglu) {
                 for (int i = et; i < BLOCK_N; i += kEpiThreads) {
                     int col;
                     if (EPI == kEpiSwiglu) col = (i < 128) ? (n0 + i) : (p.swiglu_h + n0 + i - 128);
@@ -893,19 +870,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
                                    static_cast<uint32_t>(acc * BLOCK_N);
 
-            float st_m = -INFINITY, st_s = 0.0f;  // kEpiStoreStats: this thread's row statistics
 #pragma unroll 1
             for (int c = 0; c < STEPS; ++c, ++gstep) {
                 const uint32_t slot = gstep % SLOTS;
                 const uint32_t buf = stg0 + slot * Cfg::BUFS_PER_STEP * kStgBytes;
 
-                if (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiGelu) {
+                if (EPI == kEpiStore) {
                     // this thread: columns [c*64 + hf*32, +32) of its row
                     const int col0 = c * 64 + hf * 32;
                     uint32_t r[32];
                     ptx::tmem_ld_32x32_wait(t_acc + col0, r);
                     if (c == STEPS - 1) release_acc(acc);  // accumulator fully read
-                    float sv[EPI == kEpiStoreStats ? 32 : 1];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         float4 b0, b1;
@@ -917,47 +892,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         z[1] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 2], r[j * 8 + 3]), al, ptx::make_f2(b0.z, b0.w));
                         z[2] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 4], r[j * 8 + 5]), al, ptx::make_f2(b1.x, b1.y));
                         z[3] = ptx::fma2(ptx::make_f2_bits(r[j * 8 + 6], r[j * 8 + 7]), al, ptx::make_f2(b1.z, b1.w));
-                        const uint32_t pos = chunk_pos(hf * 4 + j);
-                        if (EPI == kEpiGelu) {
-                            ptx::st_shared_v4(buf + kStgBytes + pos, pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),
-                                              pack_f2_bf16x2(z[2]), pack_f2_bf16x2(z[3]));
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) z[k] = gelu_fwd2(z[k]);
-                        }
-                        const uint32_t w0 = pack_f2_bf16x2(z[0]), w1 = pack_f2_bf16x2(z[1]),
-                                       w2 = pack_f2_bf16x2(z[2]), w3 = pack_f2_bf16x2(z[3]);
-                        ptx::st_shared_v4(buf + pos, w0, w1, w2, w3);
-                        if (EPI == kEpiStoreStats) {  // keep the eight stored (rounded) values
-                            sv[j * 8 + 0] = ptx::bf16_lo(w0); sv[j * 8 + 1] = ptx::bf16_hi(w0);
-                            sv[j * 8 + 2] = ptx::bf16_lo(w1); sv[j * 8 + 3] = ptx::bf16_hi(w1);
-                            sv[j * 8 + 4] = ptx::bf16_lo(w2); sv[j * 8 + 5] = ptx::bf16_hi(w2);
-                            sv[j * 8 + 6] = ptx::bf16_lo(w3); sv[j * 8 + 7] = ptx::bf16_hi(w3);
-                        }
-                    }
-                    if (EPI == kEpiStoreStats) {
-                        // online softmax statistics of this thread's 32 stored values: running
-                        // maximum st_m and sum of exp(value - st_m), columns >= v_real left out
-                        const int g0 = n0 + col0;
-                        float mx = -INFINITY;
-                        if (g0 + 32 > p.v_real) {  // only the tile that straddles v_real masks
-#pragma unroll
-                            for (int k = 0; k < 32; ++k)
-                                if (g0 + k >= p.v_real) sv[k] = -INFINITY;
-                        }
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) mx = fmaxf(mx, sv[k]);
-                        if (mx > st_m) {
-                            st_s *= exp2f((st_m - mx) * 1.4426950408889634f);  // 0 while st_m = -inf
-                            st_m = mx;
-                        }
-                        if (st_m > -INFINITY) {
-                            const float ms = st_m * 1.4426950408889634f;
-                            float acc_s = 0.0f;
-#pragma unroll
-                            for (int k = 0; k < 32; ++k)
-                                acc_s += ptx::ex2_approx(fmaf(sv[k], 1.4426950408889634f, -ms));
-                            st_s += acc_s;
-                        }
+                        ptx::st_shared_v4(buf + chunk_pos(hf * 4 + j), pack_f2_bf16x2(z[0]), pack_f2_bf16x2(z[1]),
+                                          pack_f2_bf16x2(z[2]), pack_f2_bf16x2(z[3]));
                     }
                 } else if (EPI == kEpiSwiglu) {
                     // step c covers out columns [c*64, +64): gate TMEM cols c*64.., up cols 128 + c*64..
@@ -987,37 +923,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                           ptx::pack_bf16x2(uu[2], uu[3]), ptx::pack_bf16x2(uu[4], uu[5]),
                                           ptx::pack_bf16x2(uu[6], uu[7]));
                     }
-                } else if (EPI == kEpiMulGeluGrad) {
-                    constexpr uint32_t NAUX = Cfg::NAUX > 0 ? Cfg::NAUX : 1;
-                    const uint32_t aslot = gstep % NAUX;
-                    const uint32_t abuf = smem + Cfg::OFF_AUX + aslot * kStgBytes;
-                    bool aok = true;
-                    if (lane == 0)
-                        aok = wait_barrier(wctx, aux_bar(static_cast<int>(aslot)), (gstep / NAUX) & 1u,
-                                           500 + static_cast<int>(aslot));
-                    aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
-                    if (!aok) {
-                        ptx::st_shared_u32_volatile(epi_abort_addr, 1);
-                        ok = false;
-                    }
-                    const int col0 = c * 64 + hf * 32;
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32_wait(t_acc + col0, r);
-                    if (c == STEPS - 1) release_acc(acc);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t cp = chunk_pos(hf * 4 + j);
-                        uint32_t x[4];
-                        ptx::ld_shared_v4(abuf + cp, x[0], x[1], x[2], x[3]);
-                        uint32_t w[4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const ptx::f2 a2 = ptx::make_f2_bits(r[j * 8 + 2 * k], r[j * 8 + 2 * k + 1]);
-                            const ptx::f2 x2 = ptx::make_f2_bits(x[k] << 16, x[k] & 0xffff0000u);
-                            w[k] = pack_f2_bf16x2(mul_gelu_bwd2(a2, x2));
-                        }
-                        ptx::st_shared_v4(buf + cp, w[0], w[1], w[2], w[3]);
-                    }
                 } else {  // kEpiF32: 32 fp32 columns per step, 16 per thread
                     uint32_t r[16];
                     ptx::tmem_ld_32x16_wait(t_acc + c * 32 + hf * 16, r);
@@ -1040,15 +945,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                   if (ptx::elect_one()) {
                     const int y = m0;
                     if (ok && y < p.M) {
-                        if (EPI == kEpiStore || EPI == kEpiStoreStats || EPI == kEpiMulGeluGrad) {
+                        if (EPI == kEpiStore) {
                             const int x = n0 + c * 64;
                             if (x < p.N) ptx::tma_store_2d(&tmD, buf, x, y);
-                        } else if (EPI == kEpiGelu) {
-                            const int x = n0 + c * 64;
-                            if (x < p.N) {
-                                ptx::tma_store_2d(&tmD, buf, x, y);
-                                ptx::tma_store_2d(&tmE, buf + kStgBytes, x, y);
-                            }
                         } else if (EPI == kEpiSwiglu) {
                             const int x = n0 + c * 64;
                             if (x < p.swiglu_h) {
@@ -1065,18 +964,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                         }
                     }
                     ptx::bulk_commit_group();
-                    // every thread has read this step's pre-activation buffer (barrier above): refill it
-                    if (EPI == kEpiMulGeluGrad) issue_aux(gstep + AUX_AHEAD);
                     if (SLOTS == 1) ptx::bulk_wait_group_read<0>();
                   }
                 }
                 __syncwarp();  // the single-lane block above rejoins its warp before collective ops
                 if (SLOTS == 1) ptx::named_bar_sync(1, kEpiThreads);
-            }
-            if (EPI == kEpiStoreStats) {
-                const long long grow = static_cast<long long>(m0) + row;
-                if (ok && grow < p.M)
-                    p.stats[grow * p.stats_ld + n_blk * 2 + hf] = make_float2(st_m, st_s);
             }
             if (++acc == 2) {
                 acc = 0;

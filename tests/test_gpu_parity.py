@@ -609,3 +609,40 @@ def test_results_beyond_two_to_the_31_elements():
     rw = oracle.linear_backward(f32(dl[:, ot]), f32(inp), f32(w[ot]), want=("dweight",))
     check_f32(dw[ot], rw["dweight"], "dweight rows")
     assert torch.all(dw[V:] == 0)
+
+
+@pytest.mark.parametrize("model,config_id", [("gpt2_block", 2), ("gpt2", 4), ("qwen3", 5)])
+def test_graph_replay_of_a_step_equals_the_eager_step(model, config_id):
+    """bench.py times a captured CUDA graph of the step: the replay must produce what the eager
+    launches produce (outputs and dinp bit for bit, the atomically accumulated gradients to rounding)
+    with programmatic dependent launch on, both for the own-activation backward (config 2) and the
+    chained fc -> proj form with the fused GELU backward (config 4)."""
+    from paper_2609_28568_b200.stack import LinearStack
+    BT = 2048 if model == "gpt2_block" else 1024
+    a = LinearStack(model, BT=BT, micro_steps=3, device=DEV, config_id=config_id)
+    a.step()
+    b = LinearStack(model, BT=BT, micro_steps=3, device=DEV, config_id=config_id)
+    b.step()  # warm-up: workspace and tensor maps exist before the capture
+    for L in b.layers:
+        L.dweight.fill_(7.0)
+        if L.dbias is not None:
+            L.dbias.fill_(7.0)
+        L.dinp.zero_()
+        L.out.zero_()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cap):
+            b.step()
+    torch.cuda.current_stream().wait_stream(cap)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    for La, Lb in zip(a.layers, b.layers):
+        assert torch.equal(Lb.out, La.out), La.spec.name
+        assert torch.equal(Lb.dinp, La.dinp), La.spec.name
+        assert rel_frob(f32(Lb.dweight[:64]), f32(La.dweight[:64])) < 1e-5, La.spec.name
+        assert rel_frob(f32(Lb.dweight[-64:]), f32(La.dweight[-64:])) < 1e-5, La.spec.name
+        if La.dbias is not None:
+            assert rel_frob(f32(Lb.dbias), f32(La.dbias)) < 1e-5, La.spec.name

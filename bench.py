@@ -118,11 +118,11 @@ def oracle_sample(seconds_hint: float = 15.0):
     import oracle
     from paper_2609_28568_b200 import shapes, synth
 
-    BT = 8192
+    BT, HEAD_ROWS = 16384, 4096  # about 12 s of work on 16 cores
     specs = shapes.gpt2_block() + [shapes.gpt2_lm_head()]
     flops, secs = 0, 0.0
     for li, s in enumerate(specs):
-        rows = BT if s.OC != shapes.VOCAB_PADDED else 1024
+        rows = BT if s.OC != shapes.VOCAB_PADDED else HEAD_ROWS
         f = lambda t: t.float().numpy()
         inp = f(synth.normal(9000 + li, (rows, s.C), 1.0))
         w = f(synth.normal(9100 + li, (s.OC, s.C), s.w_std))
@@ -135,7 +135,7 @@ def oracle_sample(seconds_hint: float = 15.0):
         secs += time.perf_counter() - t0
         flops += 6 * rows * s.C * s.OC
     desc = (f"fp32 oracle on one GPT-2 block (qkv, attn-proj, fc+GELU, proj) fwd+bwd at BT={BT} and the "
-            f"tied head fwd+bwd on 1024 rows; {flops / 1e9:.1f} GFLOP")
+            f"tied head fwd+bwd on {HEAD_ROWS} rows; {flops / 1e9:.1f} GFLOP")
     return flops, secs, desc, oracle.num_threads()
 
 

@@ -272,6 +272,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from the host in the timed region instead of replaying a CUDA graph")
+    ap.add_argument("--one-stream", action="store_true",
+                    help="keep the weight-gradient calls on the main stream (default: a second stream)")
     ap.add_argument("--dp", action="store_true",
                     help="data parallel instead of replicas: the same weights on every rank, its own rows, and "
                          "the fp32 gradients all-reduced (NCCL) in buckets under the last micro-step's backward; "
@@ -308,8 +310,10 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     model, BT, micro_steps, cfg_id, wgrad, wdesc = WORKLOADS[args.workload]
+    # weight gradients on a second stream (not with --dp: the reducer's events follow one stream)
     stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
-                        wgrad=wgrad, shared_weights=args.dp)
+                        wgrad=wgrad, shared_weights=args.dp,
+                        wgrad_stream=not (args.dp or args.one_stream))
     reducer = None
     if args.dp:
         from paper_2609_28568_b200 import dp as dpmod
@@ -487,6 +491,7 @@ def main():
             "config": {"workload": args.workload, "description": wdesc, "BT": BT,
                        "micro_steps": micro_steps, "l2": "inputs_exceed_l2 (a step touches >20 GB)",
                        "launch": "eager" if args.no_graph else "cuda_graph_replay",
+                       "streams": 2 if stack.wgrad_stream else 1,
                        "parallelism": (f"dp{world}: fp32 gradient all-reduce in {len(reducer.b.buckets)} buckets "
                                        f"under the last micro-step's backward" if reducer is not None
                                        else f"replicas x{world}, no collective")},

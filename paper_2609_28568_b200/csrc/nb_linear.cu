@@ -286,7 +286,22 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attrs[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
-    cfg.numAttrs = g_use_pdl ? 2 : 1;
+    // While a stream is being captured into a graph, a launch that follows a wait on another
+    // stream has more than one dependency; with the programmatic attribute all of them became
+    // programmatic edges and the kernel then waited for only one (observed: a consumer started
+    // before its cross-stream producer had finished). Such a launch keeps full dependencies.
+    bool pdl = g_use_pdl;
+    if (pdl) {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        const cudaGraphNode_t *deps = nullptr;
+        size_t ndeps = 0;
+        if (cudaStreamGetCaptureInfo(stream, &cs, nullptr, nullptr, &deps, &ndeps) != cudaSuccess) {
+            (void)cudaGetLastError();
+            cs = cudaStreamCaptureStatusNone;
+        }
+        if (cs == cudaStreamCaptureStatusActive && ndeps != 1) pdl = false;
+    }
+    cfg.numAttrs = pdl ? 2 : 1;
     NB_CUDA(cudaLaunchKernelEx(&cfg, gemm_kernel<Cfg>, tA, tB, tD, tE, tA2, tB2, p));
     ++g_launches;
     return NB_OK;

@@ -40,7 +40,7 @@ class _Layer:
 class LinearStack:
     def __init__(self, model: str, BT: int, micro_steps: int, device="cuda", config_id: int = 4,
                  seed_offset: int = 0, wgrad: bool = True, generate: bool = True,
-                 shared_weights: bool = False):
+                 shared_weights: bool = False, wgrad_stream: bool = False):
         self.model, self.BT, self.micro_steps, self.device = model, BT, micro_steps, device
         self.wgrad = wgrad
         self.layers: list[_Layer] = []
@@ -71,6 +71,12 @@ class LinearStack:
         # data parallel: every rank holds the same weights and its own rows (seed_offset = rank
         # then only moves the activations and output gradients); replicas differ in everything
         self.shared_weights = shared_weights
+        # Weight-gradient calls on a second stream: dgrad of the layer below needs only this layer's
+        # dgrad, so the two chains are independent, and the CTAs of one chain's next kernel take the
+        # SMs that the other chain's kernel leaves idle in its last wave and tail.
+        self.wgrad_stream = bool(wgrad_stream and wgrad)
+        self._side = None
+        self._wg_done = {}   # layer index -> event: its last weight-gradient call on the side stream
         self._allocate()
         if generate:
             self.generate_inputs()
@@ -150,6 +156,11 @@ class LinearStack:
         BT = self.BT
         for L in self.layers:
             s = L.spec
+            # a consumer chained to this layer read L.out in its weight-gradient call on the side
+            # stream during the previous micro-step: that read precedes this rewrite of L.out
+            ev = self._wg_done.pop(("out", L.index), None)
+            if ev is not None:
+                torch.cuda.current_stream().wait_event(ev)
             if hook:
                 hook("fwd", L, True)
             nb.nb_linear_forward_ex(L.out, L.pre, self.layer_inp(L, ms), L.weight, L.bias, BT, s.C,
@@ -157,7 +168,67 @@ class LinearStack:
             if hook:
                 hook("fwd", L, False)
 
+    def _backward_two_streams(self, ms: int):
+        """dgrad calls on the current stream, dweight / dbias calls on the side stream. Every buffer
+        that one stream writes and the other reads is ordered by an event: the forward outputs and
+        the dz a fused dgrad produces (read by side-stream calls), and, in the other direction, the
+        rewrite of those buffers in the next micro-step."""
+        BT = self.BT
+        acc = 1 if ms > 0 else 0
+        main = torch.cuda.current_stream()
+        if self._side is None:
+            self._side = torch.cuda.Stream(device=self.device)
+        side = self._side
+        ev = torch.cuda.Event()
+        ev.record(main)          # this micro-step's forward (and the inputs it was given) precede it
+        side.wait_event(ev)
+        for L in reversed(self.layers):
+            s = L.spec
+            if L.dz_from is not None:
+                dout, act, pre = L.dz_from.dinp, shapes.ACT_NONE, None
+            else:
+                dout, act, pre = L.dout[ms], s.act, L.pre
+            inp_pre = L.chained_from.pre if L.chained_from else None
+            if act != shapes.ACT_NONE:
+                # own-activation backward forms dz in the library's one scratch buffer: both
+                # products stay in one call on the current stream (always the same stream per layer)
+                nb.nb_linear_backward_ex(L.dinp, L.dweight, L.dbias, dout, self.layer_inp(L, ms), L.weight,
+                                         pre, inp_pre, BT, s.C, s.OC, act, acc)
+                continue
+            # this dgrad rewrites L.dinp, which the producer's side-stream call of the previous
+            # micro-step read as its dz
+            evd = self._wg_done.pop(("dinp", L.index), None)
+            if evd is not None:
+                main.wait_event(evd)
+            nb.nb_linear_backward_ex(L.dinp, None, None, dout, self.layer_inp(L, ms), L.weight, pre, inp_pre,
+                                     BT, s.C, s.OC, act, acc)
+            if L.chained_from is not None:
+                # this dgrad wrote the dz that the producer's weight gradient reads
+                e2 = torch.cuda.Event()
+                e2.record(main)
+                side.wait_event(e2)
+            with torch.cuda.stream(side):
+                nb.nb_linear_backward_ex(None, L.dweight, L.dbias, dout, self.layer_inp(L, ms), L.weight, pre,
+                                         None, BT, s.C, s.OC, act, acc)
+                if L.chained_from is not None or L.dz_from is not None:
+                    e3 = torch.cuda.Event()
+                    e3.record(side)
+                    if L.chained_from is not None:   # read the producer's out
+                        self._wg_done[("out", L.chained_from.index)] = e3
+                    if L.dz_from is not None:        # read the consumer's dinp
+                        self._wg_done[("dinp", L.dz_from.index)] = e3
+
+    def join(self):
+        """The current stream waits for the weight-gradient stream (no-op without one)."""
+        if self._side is not None:
+            e = torch.cuda.Event()
+            e.record(self._side)
+            torch.cuda.current_stream().wait_event(e)
+            self._wg_done.clear()
+
     def backward(self, ms: int, hook=None):
+        if self.wgrad_stream and hook is None:
+            return self._backward_two_streams(ms)
         BT = self.BT
         acc = 1 if ms > 0 else 0
         for L in reversed(self.layers):
@@ -178,11 +249,14 @@ class LinearStack:
     def micro_step(self, ms: int, hook=None):
         self.forward(ms, hook)
         self.backward(ms, hook)
+        self.join()
 
     def step(self, hook=None):
         """One pass of the whole path: every micro-step, forward then backward."""
         for ms in range(self.micro_steps):
-            self.micro_step(ms, hook)
+            self.forward(ms, hook)
+            self.backward(ms, hook)
+        self.join()
 
     # ------------------------------------------------------------------ data parallel
     def attach_gradient_buckets(self, bucket_bytes: int = 32 << 20):

@@ -646,3 +646,44 @@ def test_graph_replay_of_a_step_equals_the_eager_step(model, config_id):
         assert rel_frob(f32(Lb.dweight[-64:]), f32(La.dweight[-64:])) < 1e-5, La.spec.name
         if La.dbias is not None:
             assert rel_frob(f32(Lb.dbias), f32(La.dbias)) < 1e-5, La.spec.name
+
+
+@pytest.mark.parametrize("model,config_id", [("gpt2_block", 2), ("gpt2", 4), ("qwen3", 5)])
+def test_weight_gradients_on_a_second_stream_match_the_single_stream_step(model, config_id):
+    """The stack driver's two-stream backward (dgrad chain on one stream, dweight / dbias on another)
+    orders every buffer the two streams share: same gradients, outputs and dinp as the single-stream
+    step, eagerly and when the step is replayed from a captured CUDA graph (where a launch that
+    follows a cross-stream wait gives up programmatic dependent launch)."""
+    from paper_2609_28568_b200.stack import LinearStack
+    BT = 2048 if model == "gpt2_block" else 1024
+    a = LinearStack(model, BT=BT, micro_steps=3, device=DEV, config_id=config_id)
+    a.step()
+    b = LinearStack(model, BT=BT, micro_steps=3, device=DEV, config_id=config_id, wgrad_stream=True)
+    b.step()
+    torch.cuda.synchronize()
+
+    def same(tag):
+        for La, Lb in zip(a.layers, b.layers):
+            assert rel_frob(f32(Lb.dweight[:64]), f32(La.dweight[:64])) < 1e-5, (tag, La.spec.name)
+            assert rel_frob(f32(Lb.dweight[-64:]), f32(La.dweight[-64:])) < 1e-5, (tag, La.spec.name)
+            if La.dbias is not None:
+                assert rel_frob(f32(Lb.dbias), f32(La.dbias)) < 1e-5, (tag, La.spec.name)
+            assert torch.equal(Lb.dinp, La.dinp), (tag, La.spec.name)
+            assert torch.equal(Lb.out, La.out), (tag, La.spec.name)
+    same("eager")
+    for L in b.layers:
+        L.dweight.fill_(7.0)
+        if L.dbias is not None:
+            L.dbias.fill_(7.0)
+        L.dinp.zero_()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cap):
+            b.step()
+    torch.cuda.current_stream().wait_stream(cap)
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    same("graph")

@@ -456,7 +456,8 @@ def main():
         "frac": achieved_tf / peak_tf, "traffic": traffic,
         "peak_source": f"{peak_src} cuBLAS bf16 ({'sustained' if long_step else 'burst'})",
         "kernel": "nb::gemm_kernel (tcgen05 fwd / dgrad / wgrad instantiations): every launch of a step; "
-                  "average launch duration = timed region (CUDA events on the launch stream) / launches; "
+                  "average launch duration = timed region (CUDA events on the launch stream) / launches "
+                  "(with two streams the ends of launches overlap); "
                   "per_call from a second pass over the same steps with an event at every call boundary",
         "launches_per_step": launches / args.steps,
         "avg_launch_us": my_ms_per_step * 1e3 / (launches / args.steps) if launches else None,

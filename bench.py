@@ -38,6 +38,9 @@ WORKLOADS = {
     "qwen3_adapter": ("qwen3", 16384, 1, 5, True, "Qwen3-0.6B-shaped linears x28, B=8 T=2048 (config 5a)"),
     "qwen3_adapter_frozen": ("qwen3", 16384, 1, 5, False,
                              "Qwen3-0.6B-shaped linears x28, frozen base: fwd+dgrad (config 5b)"),
+    "qwen3_lora": ("qwen3_lora", 16384, 1, 6, False,
+                   "Qwen3-0.6B's seven projections x28 with rank-16 adapters (alpha 32, rank-stabilised), "
+                   "frozen base: fwd, dinp, dA, dB, B=8 T=2048"),
 }
 
 
@@ -311,9 +314,15 @@ def main():
 
     model, BT, micro_steps, cfg_id, wgrad, wdesc = WORKLOADS[args.workload]
     # weight gradients on a second stream (not with --dp: the reducer's events follow one stream)
-    stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
-                        wgrad=wgrad, shared_weights=args.dp,
-                        wgrad_stream=not (args.dp or args.one_stream))
+    if model == "qwen3_lora":
+        from paper_2609_28568_b200.stack import LoraStack
+        if args.dp:
+            raise SystemExit("--dp is wired for the dense stacks only")
+        stack = LoraStack(BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank)
+    else:
+        stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
+                            wgrad=wgrad, shared_weights=args.dp,
+                            wgrad_stream=not (args.dp or args.one_stream))
     reducer = None
     if args.dp:
         from paper_2609_28568_b200 import dp as dpmod

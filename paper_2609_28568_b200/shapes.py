@@ -65,6 +65,19 @@ def qwen3_block() -> list[LinearSpec]:
     ]
 
 
+def qwen3_lora_projections() -> list[LinearSpec]:
+    """The seven adapted projections of a Qwen3-0.6B layer (no bias, no fused activation)."""
+    return [
+        LinearSpec("q", 1024, 2048, False),
+        LinearSpec("k", 1024, 1024, False),
+        LinearSpec("v", 1024, 1024, False),
+        LinearSpec("o", 2048, 1024, False),
+        LinearSpec("gate", 1024, 3072, False),
+        LinearSpec("up", 1024, 3072, False),
+        LinearSpec("down", 3072, 1024, False),
+    ]
+
+
 def gpt2_param_count() -> tuple[int, int]:
     """(parameters, tensors) of GPT-2 124M with the real vocabulary, tied head."""
     C, L = GPT2_CHANNELS, GPT2_LAYERS

@@ -297,3 +297,103 @@ class LinearStack:
             self.forward(ms, hook)
             self.backward(ms, on_call if ms == last else hook)
         reducer.finish()
+
+
+class LoraStack:
+    """The adapter stage's linears (paper: Method/The clinical stage): Qwen3-0.6B's seven projections
+    per layer, base weights frozen, a rank-r adapter beside each (rank-stabilised scale alpha / sqrt(r)).
+    A step is every adapted projection forward, then backward in reverse order: dinp through the frozen
+    weight and the adapter, fp32 gradients of A and B accumulated over the micro-steps. Same interface
+    as `LinearStack` as far as the benchmark uses it."""
+
+    def __init__(self, BT: int, micro_steps: int = 1, device="cuda", r: int = 16, alpha: float = 32.0,
+                 layers: int = shapes.QWEN3_LAYERS, config_id: int = 6, seed_offset: int = 0,
+                 generate: bool = True):
+        self.BT, self.micro_steps, self.device, self.r = BT, micro_steps, device, r
+        self.scale = alpha / (r ** 0.5)
+        self.wgrad, self.wgrad_stream = False, False
+        self.config_id, self.seed_offset = config_id, seed_offset
+        self.layers: list[_Layer] = []
+        idx = 0
+        bf, f32 = torch.bfloat16, torch.float32
+        for _ in range(layers):
+            for s in shapes.qwen3_lora_projections():
+                L = _Layer(s, idx)
+                L.weight = torch.empty((s.OC, s.C), dtype=bf, device=device)
+                L.lora_a = torch.empty((r, s.C), dtype=bf, device=device)
+                L.lora_b = torch.empty((s.OC, r), dtype=bf, device=device)
+                L.t = torch.empty((BT, r), dtype=bf, device=device)
+                L.u = torch.empty((BT, r), dtype=bf, device=device)
+                L.dlora_a = torch.empty((r, s.C), dtype=f32, device=device)
+                L.dlora_b = torch.empty((s.OC, r), dtype=f32, device=device)
+                L.out = torch.empty((BT, s.OC), dtype=bf, device=device)
+                L.dinp = torch.empty((BT, s.C), dtype=bf, device=device)
+                L.inp = [torch.empty((BT, s.C), dtype=bf, device=device) for _ in range(micro_steps)]
+                L.dout = [torch.empty((BT, s.OC), dtype=bf, device=device) for _ in range(micro_steps)]
+                self.layers.append(L)
+                idx += 1
+        if generate:
+            self.generate_inputs()
+
+    def seed(self, L, role: int, ms: int = 0) -> int:
+        return synth.tensor_seed(self.config_id, L.index, role, ms) + 100000 * self.seed_offset
+
+    def generate_inputs(self):
+        dev = self.device
+        for L in self.layers:
+            s = L.spec
+            L.weight.copy_(synth.normal(self.seed(L, 1), (s.OC, s.C), s.w_std, dev))
+            L.lora_a.copy_(synth.normal(self.seed(L, 4), (self.r, s.C), 0.02, dev))
+            L.lora_b.copy_(synth.normal(self.seed(L, 5), (s.OC, self.r), 0.02, dev))  # a trained adapter
+            for ms in range(self.micro_steps):
+                L.inp[ms].copy_(synth.normal(self.seed(L, 0, ms), (self.BT, s.C), 1.0, dev))
+                L.dout[ms].copy_(synth.normal(self.seed(L, 3, ms), (self.BT, s.OC), 1e-3, dev))
+
+    def input_tensors(self, ms: int):
+        return [t for L in self.layers for t in (L.inp[ms], L.dout[ms])]
+
+    def gradient_tensors(self):
+        return [g for L in self.layers for g in (L.dlora_a, L.dlora_b)]
+
+    def flops_per_micro_step(self) -> int:
+        """Forward and dinp through the frozen weight, and the six rank-r products of a projection."""
+        return sum(4 * self.BT * L.spec.C * L.spec.OC + 6 * self.BT * self.r * (L.spec.C + L.spec.OC)
+                   for L in self.layers)
+
+    def calls_per_micro_step(self) -> int:
+        return 2 * len(self.layers)
+
+    def layer_inp(self, L, ms: int):
+        return L.inp[ms]
+
+    def forward(self, ms: int, hook=None):
+        for L in self.layers:
+            s = L.spec
+            if hook:
+                hook("fwd", L, True)
+            nb.nb_lora_linear_forward(L.out, L.t, L.inp[ms], L.weight, None, L.lora_a, L.lora_b, self.scale,
+                                      self.BT, s.C, s.OC, self.r)
+            if hook:
+                hook("fwd", L, False)
+
+    def backward(self, ms: int, hook=None):
+        acc = 1 if ms > 0 else 0
+        for L in reversed(self.layers):
+            s = L.spec
+            if hook:
+                hook("bwd", L, True)
+            nb.nb_lora_linear_backward(L.dinp, L.dlora_a, L.dlora_b, L.u, L.dout[ms], L.inp[ms], L.weight,
+                                       L.lora_a, L.lora_b, L.t, self.scale, self.BT, s.C, s.OC, self.r, acc)
+            if hook:
+                hook("bwd", L, False)
+
+    def join(self):
+        pass
+
+    def micro_step(self, ms: int, hook=None):
+        self.forward(ms, hook)
+        self.backward(ms, hook)
+
+    def step(self, hook=None):
+        for ms in range(self.micro_steps):
+            self.micro_step(ms, hook)

@@ -166,3 +166,31 @@ def test_adapter_workload_full_batch_sampled(C, OC):
                                              want_dinp=False)
     check_f32(dA, dA_ref, "dlora_a")
     check_f32(dB, dB_ref, "dlora_b")
+
+
+def test_adapter_stack_driver_two_micro_steps():
+    """The adapter-stage driver: one Qwen3 layer's seven adapted projections, two micro-steps; outputs
+    and dinp of the last micro-step and the accumulated adapter gradients against the oracle."""
+    from paper_2609_28568_b200.stack import LoraStack
+    BT = 384
+    st = LoraStack(BT, micro_steps=2, device=DEV, layers=1)
+    st.step()
+    torch.cuda.synchronize()
+    assert [L.spec.name for L in st.layers] == ["q", "k", "v", "o", "gate", "up", "down"]
+    for L in st.layers:
+        w, a, b = f32(L.weight), f32(L.lora_a), f32(L.lora_b)
+        o_ref = oracle.lora_forward(f32(L.inp[1]), w, None, a, b, st.scale)
+        t_ref, _ = oracle.linear_forward(f32(L.inp[1]), a)
+        check_bf16(L.out, o_ref, L.spec.name + " out", extra=_rounding_slack(st.scale * t_ref, b.T))
+        dA = dB = None
+        for ms in range(2):
+            di_ref, dA, dB = oracle.lora_backward(f32(L.dout[ms]), f32(L.inp[ms]), w, a, b, st.scale,
+                                                  dA=dA, dB=dB, accumulate=ms > 0)
+        u_ref = oracle.linear_backward(f32(L.dout[1]), None, b, want=("dinp",))["dinp"]
+        check_bf16(L.dinp, di_ref, L.spec.name + " dinp", extra=_rounding_slack(st.scale * u_ref, a))
+        check_f32(L.dlora_a, dA, L.spec.name + " dlora_a")
+        check_f32(L.dlora_b, dB, L.spec.name + " dlora_b")
+    assert st.flops_per_micro_step() == sum(
+        4 * BT * c * oc + 6 * BT * 16 * (c + oc)
+        for c, oc in ((1024, 2048), (1024, 1024), (1024, 1024), (2048, 1024), (1024, 3072), (1024, 3072),
+                      (3072, 1024)))

@@ -540,11 +540,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         const int row = q * 32 + lane;
       if constexpr (Cfg::WARP_EPI) {
         // ------------------------------------------------------------ epilogue, warp by warp
-        // A warp owns 32 rows (its TMEM lane quarter) x 128 columns (its half) of the tile. It reads
-        // them from TMEM 32 columns at a time (the next load in flight while it works on the
-        // current one), applies the epilogue, stages 32 x 64 boxes in its own 4 KB buffers and
-        // stores them with its own TMA copies. No barrier joins the warps: while one waits for
-        // TMEM, a proxy fence or a store, the others compute.
+        // A warp owns 32 rows (its TMEM lane quarter) x 128 columns (its half) of the tile. It issues
+        // the TMEM loads of all its columns at once, then, 32 columns at a time, applies the
+        // epilogue, stages 32 x 64 boxes in its own 4 KB buffers and stores them with its own TMA
+        // copies. No barrier joins the warps: while one waits for TMEM, a proxy fence or a store,
+        // the others compute.
         const int ew = warp - 2;                  // 0..7
         constexpr uint32_t kBoxBytes = 32 * 128;  // 32 rows x 64 bf16, 128-byte swizzled
         constexpr uint32_t NBUF = Cfg::WARP_BOXES;  // kEpiGelu: activated + pre-activation; kEpiF32: a ring of two

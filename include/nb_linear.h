@@ -280,6 +280,22 @@ int64_t nb_kernel_launches(void);
 int nb_debug_split_plan(int64_t M, int64_t N, int64_t K, int slots, int tile_m, int *out);
 
 /*
+ * Host-only view of how nb_linear_backward_ex schedules a layer whose dinp and fp32 dweight are
+ * both requested (BT > 128): one persistent launch whose CTA pairs each walk a list of work units,
+ * 256 x 256 tiles of dinp over all of K = OC and 256 x 256 tiles of dweight over ranges of 64-row
+ * k-blocks of K = BT (paper: Results/Speed, stage table, the GEMM row: this is its backward half
+ * for one layer). No device is touched. `pairs` is the number of CTA pairs (SM count / 2),
+ * `gelu_grad` whether the producer's GELU derivative is applied in the dinp epilogue (it makes
+ * those units dearer in the balance). out[0..7] = dinp row tiles, dinp column tiles, k-blocks of
+ * a dinp tile, dweight row tiles, dweight column tiles, k-blocks of K = BT, k-blocks per dweight
+ * chunk, whole rounds. Then one record of six ints per unit in execution order of each pair:
+ * (pair, is_dweight, row tile, column tile, first k-block, end k-block). Returns the number of
+ * records, or minus an NB_ERR_* code (buffer too small, shape the schedule does not cover).
+ */
+int nb_debug_layer_bwd_plan(int64_t BT, int64_t C, int64_t OC, int pairs, int gelu_grad, int *out,
+                            int64_t cap);
+
+/*
  * Self-test of the bounded-wait mechanism: launches a one-block kernel that waits, for
  * at most `limit_us` microseconds, on a barrier nothing ever signals, then returns
  * normally after recording the expiry. nb_check_status() afterwards reports

@@ -24,7 +24,7 @@ EXPORTS = (
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
     "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
     "nb_debug_split_plan", "nb_cast_f32_to_bf16", "nb_lm_head_ce_forward", "nb_ce_backward",
-    "nb_lora_linear_forward", "nb_lora_linear_backward",
+    "nb_lora_linear_forward", "nb_lora_linear_backward", "nb_debug_layer_bwd_plan",
 )
 
 _lib = None
@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         L.nb_lm_head_ce_forward.argtypes = [_vp] * 6 + [_i64] * 4 + [_vp]
         L.nb_ce_backward.argtypes = [_vp] * 4 + [ctypes.c_float] + [_i64] * 3 + [_vp]
         L.nb_debug_split_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int)]
+        L.nb_debug_layer_bwd_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int), _i64]
         _lib = L
     return _lib
 
@@ -197,6 +198,19 @@ def nb_debug_split_plan(M: int, N: int, K: int, slots: int, tile_m: int):
     out = (_int * 5)()
     _check(lib().nb_debug_split_plan(M, N, K, slots, tile_m, out))
     return tuple(out)
+
+
+def nb_debug_layer_bwd_plan(BT: int, C: int, OC: int, pairs: int, gelu_grad: bool):
+    """(header of eight ints, list of (pair, is_dweight, row tile, column tile, kb0, kb1)) of the
+    one-launch layer backward; raises NbError for shapes its schedule does not cover."""
+    cap = 8 + 6 * (4 * pairs + 64 + 2 * (-(-BT // 256)) * (-(-C // 256))
+                   + 2 * (-(-OC // 256)) * (-(-C // 256)) * max(1, BT // 1024))
+    out = (_int * cap)()
+    n = lib().nb_debug_layer_bwd_plan(BT, C, OC, pairs, int(bool(gelu_grad)), out, cap)
+    if n < 0:
+        raise NbError(-n, lib().nb_last_error().decode())
+    recs = [tuple(out[8 + 6 * i: 14 + 6 * i]) for i in range(n)]
+    return tuple(out[:8]), recs
 
 
 def nb_kernel_launches() -> int:

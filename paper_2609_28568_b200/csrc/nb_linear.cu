@@ -16,6 +16,7 @@
 
 #include "elementwise.cuh"
 #include "gemm_sm100.cuh"
+#include "layer_bwd_sm100.cuh"
 
 namespace {
 
@@ -170,6 +171,21 @@ int check_dims(int64_t BT, int64_t C, int64_t OC)
     return NB_OK;
 }
 
+// Programmatic dependent launch is used unless it is switched off, or the stream is being captured
+// and this launch has more than one dependency (see launch_gemm).
+bool dependent_launch_allowed(cudaStream_t stream)
+{
+    if (!g_use_pdl) return false;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    const cudaGraphNode_t *deps = nullptr;
+    size_t ndeps = 0;
+    if (cudaStreamGetCaptureInfo(stream, &cs, nullptr, nullptr, &deps, &ndeps) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cs = cudaStreamCaptureStatusNone;
+    }
+    return !(cs == cudaStreamCaptureStatusActive && ndeps != 1);
+}
+
 // ----------------------------------------------------------------------------- GEMM launch
 struct GemmArgs {
     const void *A;  uint64_t a_rows, a_cols;   // global tensor of the A operand (bf16)
@@ -290,18 +306,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     // stream has more than one dependency; with the programmatic attribute all of them became
     // programmatic edges and the kernel then waited for only one (observed: a consumer started
     // before its cross-stream producer had finished). Such a launch keeps full dependencies.
-    bool pdl = g_use_pdl;
-    if (pdl) {
-        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-        const cudaGraphNode_t *deps = nullptr;
-        size_t ndeps = 0;
-        if (cudaStreamGetCaptureInfo(stream, &cs, nullptr, nullptr, &deps, &ndeps) != cudaSuccess) {
-            (void)cudaGetLastError();
-            cs = cudaStreamCaptureStatusNone;
-        }
-        if (cs == cudaStreamCaptureStatusActive && ndeps != 1) pdl = false;
-    }
-    cfg.numAttrs = pdl ? 2 : 1;
+    cfg.numAttrs = dependent_launch_allowed(stream) ? 2 : 1;
     NB_CUDA(cudaLaunchKernelEx(&cfg, gemm_kernel<Cfg>, tA, tB, tD, tE, tA2, tB2, p));
     ++g_launches;
     return NB_OK;
@@ -453,6 +458,222 @@ int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight
     return launch_gemm_auto<WgradF32_1, WgradF32_2>(s, a, stream);
 }
 
+// ----------------------------------------------------------------------------- one launch per layer backward
+int env_int(const char *name, int dflt)
+{
+    const char *e = getenv(name);
+    return (e && *e) ? atoi(e) : dflt;
+}
+
+// The schedule of layer_bwd_kernel for P CTA pairs (layer_bwd_sm100.cuh describes the unit list).
+// Costs are counted in k-blocks of tensor-core time: a D unit costs its k-blocks plus eD (the part
+// of its epilogue the next main loop does not hide: larger with gelu'), a W unit its k-blocks plus
+// eW. Every pair should end up with the same cost.
+//  1. K = BT of the weight gradient is cut into chunks so that there are about two W units per
+//     pair, none shorter than 32 k-blocks (every unit reduce-adds a whole fp32 tile: fewer, longer
+//     units mean less traffic; in-step timings did not tell 16 to 128 k-blocks apart).
+//  2. Whole rounds (one unit per pair) are dealt first; W rounds are spread evenly among D rounds.
+//  3. The last D round is partial: pairs [0, d_tail) take one more tile. The W units left over are
+//     laid out as one line of k-blocks and cut into P ranges, shorter by one D unit's cost for the
+//     pairs that took a tail tile. If the line is too short for that, one W round is taken back.
+// Returns NB_ERR_UNSUPPORTED when the shape needs more rounds than the order mask holds.
+int plan_layer_bwd(LayerBwdParams &p, int64_t BT, int64_t C, int64_t OC, int P, bool gelu_grad)
+{
+    memset(&p, 0, sizeof(p));
+    if (P < 1 || P > kMaxPairs) return fail(NB_ERR_UNSUPPORTED, "CTA pair count %d out of range", P);
+    static const int eD_plain = env_int("NB_LB_ED", 3);
+    static const int eD_gelu = env_int("NB_LB_ED_GELU", 8);
+    static const int eW = env_int("NB_LB_EW", 3);
+    static const int kbc_forced = env_int("NB_LB_KBC", 0);
+    const int eD = gelu_grad ? eD_gelu : eD_plain;
+    p.BT = static_cast<int>(BT);
+    p.C = static_cast<int>(C);
+    p.OC = static_cast<int>(OC);
+    p.num_pairs = P;
+    p.d_tiles_m = static_cast<int>((BT + 255) / 256);
+    p.d_tiles_n = static_cast<int>((C + 255) / 256);
+    p.d_tiles = p.d_tiles_m * p.d_tiles_n;
+    p.d_kblocks = static_cast<int>((OC + kBlockK - 1) / kBlockK);
+    p.d_group_m = (p.d_tiles_n >= 64 ? 64 : p.d_tiles_n <= 4 ? 4 : 16) / 2;
+    p.w_tiles_m = static_cast<int>((OC + 255) / 256);
+    p.w_tiles_n = p.d_tiles_n;
+    p.w_tiles = p.w_tiles_m * p.w_tiles_n;
+    p.w_kblocks = static_cast<int>((BT + kBlockK - 1) / kBlockK);
+    int chunks = (2 * P + p.w_tiles - 1) / p.w_tiles;
+    const int max_chunks = p.w_kblocks / 32 > 1 ? p.w_kblocks / 32 : 1;
+    if (chunks > max_chunks) chunks = max_chunks;
+    if (chunks < 1) chunks = 1;
+    p.w_kbc = (p.w_kblocks + chunks - 1) / chunks;
+    if (kbc_forced > 0) p.w_kbc = kbc_forced < p.w_kblocks ? kbc_forced : p.w_kblocks;
+    chunks = (p.w_kblocks + p.w_kbc - 1) / p.w_kbc;
+    const long long w_units = 1ll * chunks * p.w_tiles;
+    if (w_units >= (1ll << 24) || p.d_tiles >= (1 << 24)) return fail(NB_ERR_UNSUPPORTED, "too many work units");
+    p.w_units = static_cast<int>(w_units);
+    p.d_rounds = p.d_tiles / P;
+    p.d_tail = p.d_tiles % P;
+    const double cD = p.d_kblocks + eD;
+    // the units of the last chunk may be shorter than the others: they all stay in the tail, where
+    // lengths are counted exactly
+    p.w_last_len = p.w_kblocks - (chunks - 1) * p.w_kbc;
+    const int even_units = p.w_last_len == p.w_kbc ? p.w_units : p.w_units - p.w_tiles;
+    int aW = even_units / P;
+    double b_hi = 0.0, b_lo = 0.0;  // tail k-blocks of a pair without / with a tail D tile
+    long long Rk = 0;
+    for (;; --aW) {
+        const long long tail_full = 1ll * (even_units - aW * P) * p.w_kbc;
+        Rk = tail_full + 1ll * (p.w_units - even_units) * p.w_last_len;
+        p.w_tail_full = static_cast<int>(tail_full < (1ll << 30) ? tail_full : (1ll << 30));
+        b_hi = static_cast<double>(Rk) / P + cD * p.d_tail / P;
+        b_lo = b_hi - cD;
+        const bool fits = p.d_tail == 0 ? (Rk == 0 || Rk >= 8ll * P) : b_lo >= 8.0;
+        if (fits || aW == 0) break;
+    }
+    if (Rk >= (1ll << 30)) return fail(NB_ERR_UNSUPPORTED, "weight-gradient tail too long");
+    p.w_rounds = aW;
+    const int rounds = p.d_rounds + p.w_rounds;
+    if (rounds > kLbMaxRounds) return fail(NB_ERR_UNSUPPORTED, "more than %d rounds", kLbMaxRounds);
+    p.round_is_w = 0;
+    for (int r = 0; r < rounds; ++r)
+        if (1ll * (r + 1) * aW / rounds > 1ll * r * aW / rounds) p.round_is_w |= 1ull << r;
+    // Tail ranges. Pair q's share is what levels the cost of the pairs still to be served: the
+    // k-blocks and per-piece allowances left on the line plus their fixed costs (tail D tile),
+    // divided among them, minus its own fixed cost. A range ends on a multiple of four k-blocks of
+    // its unit or at the unit's end.
+    (void)b_hi;
+    (void)b_lo;
+    const int tail_units = p.w_units - aW * P;
+    const long long full_units = p.w_tail_full / p.w_kbc;
+    auto unit_at = [&](long long x, long long &u_idx, long long &u_left) {
+        if (x < p.w_tail_full) {
+            u_idx = x / p.w_kbc;
+            u_left = p.w_kbc - x % p.w_kbc;
+        } else {
+            const long long xr = x - p.w_tail_full;
+            u_idx = full_units + xr / p.w_last_len;
+            u_left = p.w_last_len - xr % p.w_last_len;
+        }
+    };
+    long long x = 0;
+    p.w_tail_begin[0] = 0;
+    for (int q = 0; q < P; ++q) {
+        if (q == P - 1) {
+            x = Rk;
+        } else if (x < Rk) {
+            long long u_idx, u_left;
+            unit_at(x, u_idx, u_left);
+            const int pairs_left = P - q;
+            const int tail_d_left = p.d_tail > q ? p.d_tail - q : 0;
+            const double line_cost = static_cast<double>(Rk - x) + 1.0 * eW * (tail_units - u_idx) +
+                                     1.0 * eW * (pairs_left - 1);
+            double rem = (line_cost + cD * tail_d_left) / pairs_left - (q < p.d_tail ? cD : 0.0);
+            while (x < Rk && rem >= eW + 4) {
+                unit_at(x, u_idx, u_left);
+                long long take = static_cast<long long>(rem - eW);
+                if (take >= u_left) {
+                    take = u_left;
+                } else {
+                    take = take / 4 * 4;
+                    if (take <= 0) break;
+                }
+                x += take;
+                rem -= eW + take;
+                if (take < u_left) break;
+            }
+        }
+        p.w_tail_begin[q + 1] = static_cast<int>(x);
+    }
+    for (int q = P + 1; q <= kMaxPairs; ++q) p.w_tail_begin[q] = static_cast<int>(Rk);
+    return NB_OK;
+}
+
+using LayerBwdPlain = LbCfg<false, false>;
+using LayerBwdBias = LbCfg<false, true>;
+using LayerBwdGelu = LbCfg<true, false>;
+using LayerBwdGeluBias = LbCfg<true, true>;
+
+template <class Cfg>
+int launch_layer_bwd(DeviceState &s, const void *dz, const void *weight, const void *inp, void *dinp,
+                     const void *inp_pre, void *dweight, float *dbias, int64_t BT, int64_t C, int64_t OC,
+                     int accumulate, cudaStream_t stream)
+{
+    static bool attr_set[kMaxDevices] = {};
+    static int max_pairs[kMaxDevices] = {};
+    int dev = 0;
+    NB_CUDA(cudaGetDevice(&dev));
+    if (!attr_set[dev]) {
+        NB_CUDA(cudaFuncSetAttribute(layer_bwd_kernel<Cfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(Cfg::SMEM_BYTES)));
+        cudaLaunchConfig_t qc = {};
+        qc.gridDim = dim3(static_cast<unsigned>(s.num_sms));
+        qc.blockDim = dim3(kLbThreads);
+        qc.dynamicSmemBytes = Cfg::SMEM_BYTES;
+        cudaLaunchAttribute qa[1];
+        qa[0].id = cudaLaunchAttributeClusterDimension;
+        qa[0].val.clusterDim.x = 2;
+        qa[0].val.clusterDim.y = 1;
+        qa[0].val.clusterDim.z = 1;
+        qc.attrs = qa;
+        qc.numAttrs = 1;
+        int n = 0;
+        NB_CUDA(cudaOccupancyMaxActiveClusters(&n, layer_bwd_kernel<Cfg>, &qc));
+        if (n < 1) return fail(NB_ERR_CUDA, "no CTA pair of the layer-backward kernel fits on the device");
+        max_pairs[dev] = n < s.num_sms / 2 ? n : s.num_sms / 2;
+        if (max_pairs[dev] > kMaxPairs) max_pairs[dev] = kMaxPairs;
+        attr_set[dev] = true;
+    }
+    LayerBwdParams p;
+    int rc = plan_layer_bwd(p, BT, C, OC, max_pairs[dev], Cfg::GELU_GRAD);
+    if (rc != NB_OK) return rc;
+    p.dbias = Cfg::DBIAS ? dbias : nullptr;
+    p.status = s.status;
+    p.timeout_ns = kDefaultTimeoutNs;
+    CUtensorMap tDz, tW, tInp, tDinp, tPre, tDw;
+    if ((rc = get_tmap(s, &tDz, dz, BT, OC, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tW, weight, OC, C, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tInp, inp, BT, C, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tDinp, dinp, BT, C, 0, 32)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tDw, dweight, OC, C, 1, 32)) != NB_OK) return rc;
+    tPre = tDinp;
+    if (Cfg::GELU_GRAD && (rc = get_tmap(s, &tPre, inp_pre, BT, C, 0, 32)) != NB_OK) return rc;
+    // partial sums of every W unit are reduce-added, so a fresh gradient starts from zero
+    if (!accumulate) {
+        NB_CUDA(cudaMemsetAsync(dweight, 0, static_cast<size_t>(OC * C) * 4, stream));
+        if (Cfg::DBIAS) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * p.num_pairs));
+    cfg.blockDim = dim3(kLbThreads);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[2];
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = 2;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = dependent_launch_allowed(stream) ? 2 : 1;
+    NB_CUDA(cudaLaunchKernelEx(&cfg, layer_bwd_kernel<Cfg>, tDz, tW, tInp, tDinp, tPre, tDw, p));
+    ++g_launches;
+    return NB_OK;
+}
+
+// dinp, fp32 dweight and (optionally) dbias of one layer from its dz in one launch. Returns
+// NB_ERR_UNSUPPORTED (and launches nothing) for shapes the schedule does not cover; the caller
+// then issues the products one by one.
+int run_layer_bwd(DeviceState &s, const void *dz, const void *weight, const void *inp, void *dinp,
+                  const void *inp_pre, void *dweight, float *dbias, int64_t BT, int64_t C, int64_t OC,
+                  int accumulate, cudaStream_t stream)
+{
+    if (inp_pre) {
+        if (dbias) return launch_layer_bwd<LayerBwdGeluBias>(s, dz, weight, inp, dinp, inp_pre, dweight, dbias, BT, C, OC, accumulate, stream);
+        return launch_layer_bwd<LayerBwdGelu>(s, dz, weight, inp, dinp, inp_pre, dweight, dbias, BT, C, OC, accumulate, stream);
+    }
+    if (dbias) return launch_layer_bwd<LayerBwdBias>(s, dz, weight, inp, dinp, inp_pre, dweight, dbias, BT, C, OC, accumulate, stream);
+    return launch_layer_bwd<LayerBwdPlain>(s, dz, weight, inp, dinp, inp_pre, dweight, dbias, BT, C, OC, accumulate, stream);
+}
+
 }  // namespace
 
 // ================================================================================ C ABI
@@ -586,6 +807,15 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
         NB_CUDA(cudaGetLastError());
         ++g_launches;
         dz = s->workspace;
+    }
+
+    // Both products of the layer in one launch (the usual case of a training step): the weight
+    // gradient's k-blocks fill the waves the input gradient's tiles leave partly empty.
+    static const bool merged = env_int("NB_MERGED_BWD", 1) != 0;
+    if (merged && dinp && dweight && dweight_dtype == NB_DTYPE_F32 && use_pairs(static_cast<int>(BT))) {
+        rc = run_layer_bwd(*s, dz, weight, inp, dinp, inp_pre_act, dweight, static_cast<float *>(dbias), BT, C,
+                           OC, accumulate, stream);
+        if (rc != NB_ERR_UNSUPPORTED) return rc;
     }
 
     if (dinp) {  // dinp[BT, C] = dz[BT, OC] . W[OC, C]
@@ -890,6 +1120,31 @@ int nb_debug_split_plan(int64_t M, int64_t N, int64_t K, int slots, int tile_m, 
     out[3] = kps;
     out[4] = kblocks;
     return NB_OK;
+}
+
+int nb_debug_layer_bwd_plan(int64_t BT, int64_t C, int64_t OC, int pairs, int gelu_grad, int *out,
+                            int64_t cap)
+{
+    if (!out || cap < 8 || BT <= 0 || C <= 0 || OC <= 0) return -fail(NB_ERR_INVALID_ARG, "bad argument");
+    LayerBwdParams p;
+    const int rc = plan_layer_bwd(p, BT, C, OC, pairs, gelu_grad != 0);
+    if (rc != NB_OK) return -rc;
+    out[0] = p.d_tiles_m; out[1] = p.d_tiles_n; out[2] = p.d_kblocks;
+    out[3] = p.w_tiles_m; out[4] = p.w_tiles_n; out[5] = p.w_kblocks;
+    out[6] = p.w_kbc; out[7] = p.d_rounds + p.w_rounds;
+    int64_t n = 8;
+    int records = 0;
+    for (int q = 0; q < pairs; ++q) {
+        LbIter it(p, q);
+        LbUnit u;
+        while (it.next(p, u)) {
+            if (n + 6 > cap) return -fail(NB_ERR_INVALID_ARG, "output buffer too small");
+            out[n++] = q; out[n++] = u.is_w; out[n++] = u.m_blk; out[n++] = u.n_blk;
+            out[n++] = u.kb0; out[n++] = u.kb1;
+            ++records;
+        }
+    }
+    return records;
 }
 
 int nb_debug_wait_timeout(int64_t limit_us)

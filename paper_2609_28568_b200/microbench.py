@@ -4,7 +4,8 @@
 
 KIND: fwd, fwd_nobias, fwd_gelu, fwd_swiglu, dgrad, dgrad_fused (dgrad with the producer's GELU
 backward in the epilogue), wgrad (accumulating), wgrad_bias (wgrad with the fused bias gradient),
-dbias (stand-alone column reduction), bwd (dgrad + wgrad + dbias in one call), cast (fp32 -> bf16
+dbias (stand-alone column reduction), bwd (dinp + dweight + dbias in one call), bwd_nobias (dinp +
+dweight), bwd_fused (bwd with the producer's GELU backward in the dinp epilogue), cast (fp32 -> bf16
 master-weight cast of OC*C elements; reports GB/s), head_ce (head forward with the fused softmax
 statistics, vocabulary OC with the last 47 columns as padding), ce_bwd (dlogits from logits, GB/s),
 lora_fwd / lora_bwd (rank-16 adapter beside a frozen weight; TFLOP/s counts base + adapter flops).
@@ -51,6 +52,8 @@ def main(argv) -> int:
                                                        0, 1),
         "dbias": lambda: nb.nb_reduce_dbias(db, dout, BT, OC, 1),
         "bwd": lambda: nb.nb_linear_backward_ex(dinp, dw, db, dout, inp, w, None, None, BT, C, OC, 0, 1),
+        "bwd_nobias": lambda: nb.nb_linear_backward_ex(dinp, dw, None, dout, inp, w, None, None, BT, C, OC, 0, 1),
+        "bwd_fused": lambda: nb.nb_linear_backward_ex(dinp, dw, db, dout, inp, w, None, ipre, BT, C, OC, 0, 1),
     }
     if kind == "cast":
         n = OC * C
@@ -99,7 +102,7 @@ def main(argv) -> int:
     if kind == "ce_bwd":
         print(f"ce_bwd BT={BT} Vp={OC}: {ms * 1e3:.1f} us/call  {BT * OC * 4 / ms / 1e6:.1f} GB/s")
         return 0
-    flops = 2 * BT * C * OC * (2 if kind == "bwd" else 1)
+    flops = 2 * BT * C * OC * (2 if kind.startswith("bwd") else 1)
     if kind == "lora_fwd":
         flops += 2 * BT * 16 * (C + OC)
     if kind == "lora_bwd":

@@ -100,3 +100,47 @@ def test_wgrad_split_plan_covers_every_k_block_once(L):
             # the chosen factor never leaves more than a wave's worth of imbalance on big problems
             if kblocks >= 64 and tm * tn <= slots:
                 assert tm * tn * splits >= slots // 2
+
+
+def test_layer_backward_plan_covers_every_unit_once(L):
+    """Host logic of the one-launch layer backward: over all CTA pairs, every dinp tile appears once
+    with its whole K range, and every (dweight tile, k-block) is covered exactly once, whatever
+    the interleaving and the balancing cuts; loads are level across the pairs."""
+    cases = [  # BT, C, OC
+        (16384, 768, 2304), (16384, 768, 768), (16384, 768, 3072), (16384, 3072, 768),
+        (16384, 768, 50304), (4096, 768, 3072), (4096, 3072, 768), (16384, 1024, 2048),
+        (16384, 3072, 1024), (384, 768, 768), (136, 72, 200), (5000, 328, 776), (256, 8, 8),
+    ]
+    for BT, C, OC in cases:
+        for pairs in (74, 66, 1):
+            for gelu in (False, True):
+                try:
+                    hdr, recs = binding.nb_debug_layer_bwd_plan(BT, C, OC, pairs, gelu)
+                except binding.NbError as e:
+                    assert e.code == binding.NB_ERR_UNSUPPORTED and pairs == 1
+                    continue
+                dtm, dtn, dkb, wtm, wtn, wkb, kbc, rounds = hdr
+                assert (dtm, dtn, dkb) == (-(-BT // 256), -(-C // 256), -(-OC // 64))
+                assert (wtm, wtn, wkb) == (-(-OC // 256), -(-C // 256), -(-BT // 64))
+                assert 1 <= kbc <= wkb and rounds <= 64
+                d_seen = {}
+                w_cov = {}
+                load = [0] * pairs   # in the planner's cost units: k-blocks plus an allowance per unit
+                for pr, is_w, m, n, kb0, kb1 in recs:
+                    assert 0 <= pr < pairs and kb0 < kb1
+                    load[pr] += kb1 - kb0 + (3 if is_w else (8 if gelu else 3))
+                    if is_w:
+                        assert 0 <= m < wtm and 0 <= n < wtn and kb1 <= wkb
+                        cov = w_cov.setdefault((m, n), [0] * wkb)
+                        for kb in range(kb0, kb1):
+                            cov[kb] += 1
+                    else:
+                        assert 0 <= m < dtm and 0 <= n < dtn and (kb0, kb1) == (0, dkb)
+                        d_seen[(m, n)] = d_seen.get((m, n), 0) + 1
+                assert len(d_seen) == dtm * dtn and set(d_seen.values()) == {1}
+                assert len(w_cov) == wtm * wtn
+                assert all(c == [1] * wkb for c in w_cov.values())
+                if pairs > 1 and BT >= 4096:
+                    # level to within a few k-blocks (cuts are rounded to four, a cut unit pays
+                    # its allowance twice)
+                    assert max(load) - min(load) <= 16, (BT, C, OC, pairs, gelu, max(load), min(load))

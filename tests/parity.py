@@ -80,3 +80,13 @@ def sample_indices(n: int, k: int, seed: int) -> np.ndarray:
     while len(idx) < k:
         idx.add(int(rng.integers(0, n)))
     return np.array(sorted(idx), dtype=np.int64)
+
+
+def stratified_indices(n: int, box: int, seed: int) -> np.ndarray:
+    """One index in every consecutive box of `box` indices of range(n), at a seeded offset inside
+    the box: a grid of such rows and columns puts an element into every tile and every store box
+    of a result, whatever the tiling."""
+    rng = np.random.default_rng(seed)
+    starts = np.arange(0, n, box, dtype=np.int64)
+    idx = np.minimum(starts + rng.integers(0, box, size=starts.size), n - 1)
+    return np.unique(idx)

@@ -9,7 +9,7 @@ import torch
 import oracle
 from paper_2609_28568_b200 import binding as nb
 from paper_2609_28568_b200 import shapes, synth
-from parity import (Guarded, check_bf16, check_f32, f32, rel_frob, sample_indices)
+from parity import (Guarded, check_bf16, check_f32, f32, rel_frob, sample_indices, stratified_indices)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -304,6 +304,17 @@ def _fwd_sampled(name, inp, w, b, act, out, pre, seed, nrows=48, ncols=24):
     check_bf16(out[gr][:, torch.as_tensor(gc, device=DEV)], o_ref, name + " out grid")
     if pre is not None:
         check_bf16(pre[gr][:, gsel], p_ref, name + " pre grid")
+    # a stratified grid: one row in every 32-row box and one column in every 64-column box of the
+    # result, compared at their crossings, so that every tile and every 32 x 64 box an epilogue
+    # warp stores holds an element the oracle has checked
+    sr = torch.as_tensor(stratified_indices(BT, 32, seed + 4), device=DEV)
+    sc = stratified_indices(ocols, 64, seed + 5)
+    ssel = torch.as_tensor(np.concatenate([sc, sc + H]) if act == nb.ACT_SWIGLU else sc, device=DEV)
+    o_ref, p_ref = oracle.linear_forward(f32(inp[sr]), f32(w[ssel]),
+                                         f32(b[ssel]) if b is not None else None, act)
+    check_bf16(out[sr][:, torch.as_tensor(sc, device=DEV)], o_ref, name + " out stratified")
+    if pre is not None:
+        check_bf16(pre[sr][:, ssel], p_ref, name + " pre stratified")
 
 
 def _bwd_sampled(name, dz, inp, w, dinp, dw, db, seed, inp_pre=None, dw_prev=None, nrows=48, ncols=8,
@@ -334,6 +345,20 @@ def _bwd_sampled(name, dz, inp, w, dinp, dw, db, seed, inp_pre=None, dw_prev=Non
             check_f32(dw[:, ccol], ref, name + " dweight cols")
     if db is not None:
         check_f32(db, oracle.reduce_dbias(f32(dz)), name + " dbias")
+    # stratified grids (see _fwd_sampled): dinp in 32 x 64 bf16 boxes, dweight in 32 x 32 fp32 boxes
+    if dinp is not None:
+        sr = torch.as_tensor(stratified_indices(BT, 32, seed + 4), device=DEV)
+        sc = torch.as_tensor(stratified_indices(C, 64, seed + 5), device=DEV)
+        r = oracle.linear_backward(f32(dz[sr]), None, f32(w[:, sc]),
+                                   inp_pre=f32(inp_pre[sr][:, sc]) if inp_pre is not None else None,
+                                   want=("dinp",))
+        check_bf16(dinp[sr][:, sc], r["dinp"], name + " dinp stratified")
+    if dw is not None:
+        so = torch.as_tensor(stratified_indices(OC, 32, seed + 6), device=DEV)
+        sc = torch.as_tensor(stratified_indices(C, 32, seed + 7), device=DEV)
+        r = oracle.linear_backward(f32(dz[:, so]), f32(inp[:, sc]), f32(w[so][:, sc]), want=("dweight",))
+        ref = r["dweight"] + (dw_prev[so.cpu().numpy()][:, sc.cpu().numpy()] if dw_prev is not None else 0.0)
+        check_f32(dw[so][:, sc], ref, name + " dweight stratified")
 
 
 def test_config3_lm_head_full_size_sampled():
@@ -687,3 +712,117 @@ def test_weight_gradients_on_a_second_stream_match_the_single_stream_step(model,
         g.replay()
     torch.cuda.synchronize()
     same("graph")
+
+
+def _round_bf16(a: np.ndarray) -> np.ndarray:
+    """The oracle's fp64 values as the bf16 numbers a stored activation would hold."""
+    return torch.from_numpy(np.asarray(a, np.float32)).to(torch.bfloat16).float().numpy()
+
+
+@pytest.mark.parametrize("wgrad_stream", [False, True])
+def test_timed_path_block_graph_replay_matches_the_oracle(wgrad_stream):
+    """The path bench.py times (the stack driver's step inside a replayed CUDA graph, one launch per
+    layer backward on one stream or dgrad / wgrad chains on two) against the oracle as a whole:
+    one GPT-2 block, four accumulating micro-steps, fc.out feeding proj and proj's fused dgrad
+    feeding fc's backward. The last micro-step's activations and input gradients are compared with
+    the oracle fed the very buffers the GPU calls read; the accumulated weight and bias gradients
+    with the oracle's own chain over all four micro-steps, rounding to bf16 where the path stores
+    an activation (fc.out, fc.pre, proj.dinp)."""
+    from paper_2609_28568_b200.stack import LinearStack
+    BT, MS = 384, 4
+    st = LinearStack("gpt2_block", BT=BT, micro_steps=MS, device=DEV, config_id=2, wgrad_stream=wgrad_stream)
+    st.step()  # warm-up outside the capture: tensor maps and schedules exist
+    for L in st.layers:
+        L.dweight.fill_(3.0)
+        L.dbias.fill_(3.0)
+        L.out.zero_()
+        L.dinp.zero_()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cap):
+            st.step()
+    torch.cuda.current_stream().wait_stream(cap)
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    nb.nb_check_status()
+    qkv, aproj, fc, proj = st.layers
+    last = MS - 1
+    # ---- the last micro-step, call by call, on the buffers the calls read
+    for L in st.layers:
+        s = L.spec
+        x = fc.out if L is proj else L.inp[last]
+        o_ref, p_ref = oracle.linear_forward(f32(x), f32(L.weight), f32(L.bias), s.act)
+        check_bf16(L.out, o_ref, s.name + " out")
+        if L.pre is not None:
+            check_bf16(L.pre, p_ref, s.name + " pre")
+        dz = proj.dinp if L is fc else L.dout[last]
+        r = oracle.linear_backward(f32(dz), None, f32(L.weight),
+                                   inp_pre=f32(fc.pre) if L is proj else None, want=("dinp",))
+        check_bf16(L.dinp, r["dinp"], s.name + " dinp")
+    # ---- gradients accumulated over the four micro-steps
+    for L in st.layers:
+        dw_ref = np.zeros((L.spec.OC, L.spec.C))
+        db_ref = np.zeros((L.spec.OC,))
+        for ms in range(MS):
+            if L is proj:    # its input is fc's stored output of that micro-step
+                o, _ = oracle.linear_forward(f32(fc.inp[ms]), f32(fc.weight), f32(fc.bias), oracle.ACT_GELU)
+                x, dz = _round_bf16(o), f32(proj.dout[ms])
+            elif L is fc:    # its dz is proj's fused dgrad of that micro-step
+                _, pz = oracle.linear_forward(f32(fc.inp[ms]), f32(fc.weight), f32(fc.bias), oracle.ACT_GELU)
+                r = oracle.linear_backward(f32(proj.dout[ms]), None, f32(proj.weight),
+                                           inp_pre=_round_bf16(pz), want=("dinp",))
+                x, dz = f32(fc.inp[ms]), _round_bf16(r["dinp"])
+            else:
+                x, dz = f32(L.inp[ms]), f32(L.dout[ms])
+            oracle.linear_backward(dz, x, f32(L.weight), dweight=dw_ref, dbias=db_ref, accumulate=ms > 0,
+                                   want=("dweight", "dbias"))
+        check_f32(L.dweight, dw_ref, L.spec.name + " dweight over micro-steps")
+        check_f32(L.dbias, db_ref, L.spec.name + " dbias over micro-steps")
+
+
+def test_timed_path_full_stack_graph_replay_sampled_against_the_oracle():
+    """The whole GPT-2 stack driver (12 blocks and the tied head, two accumulating micro-steps) in a
+    replayed graph: the last block and the head are compared with the oracle on stratified samples
+    of every output, from the buffers the GPU calls read."""
+    from paper_2609_28568_b200.stack import LinearStack
+    BT, MS = 512, 2
+    st = LinearStack("gpt2", BT=BT, micro_steps=MS, device=DEV, config_id=4)
+    st.step()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cap):
+            st.step()
+    torch.cuda.current_stream().wait_stream(cap)
+    g.replay()
+    torch.cuda.synchronize()
+    nb.nb_check_status()
+    last = MS - 1
+    blk = st.layers[-5:-1]
+    head = st.layers[-1]
+    fc, proj = blk[2], blk[3]
+    for i, L in enumerate(blk + [head]):
+        s = L.spec
+        x = fc.out if L is proj else L.inp[last]
+        _fwd_sampled("stack " + s.name, x, L.weight, L.bias, s.act, L.out, L.pre, seed=900 + 10 * i,
+                     nrows=8, ncols=8)
+        dz = proj.dinp if L is fc else L.dout[last]
+        # the weight gradient holds both micro-steps: subtract nothing, compare the sum
+        _bwd_sampled("stack " + s.name, dz, x, L.weight, L.dinp, None, None, seed=905 + 10 * i,
+                     inp_pre=fc.pre if L is proj else None, nrows=8, ncols=4)
+        if L is not proj and L is not fc:   # inputs of both micro-steps are still in memory
+            so = torch.as_tensor(stratified_indices(s.OC, 32, 907 + 10 * i), device=DEV)
+            sc = torch.as_tensor(stratified_indices(s.C, 32, 908 + 10 * i), device=DEV)
+            ref = 0.0
+            for ms in range(MS):
+                r = oracle.linear_backward(f32(L.dout[ms][:, so]), f32(L.inp[ms][:, sc]), f32(L.weight[so][:, sc]),
+                                           want=("dweight",))
+                ref = ref + r["dweight"]
+            check_f32(L.dweight[so][:, sc], ref, "stack " + s.name + " dweight over micro-steps")
+            if L.dbias is not None:
+                ref_b = sum(oracle.reduce_dbias(f32(L.dout[ms])) for ms in range(MS))
+                check_f32(L.dbias, ref_b, "stack " + s.name + " dbias over micro-steps")

@@ -1,4 +1,4 @@
-"""The allocation-free entry point, checked against the allocating one.
+"""The allocation-free entry point, checked against the allocating one and against the oracle.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test. Users who cannot call cudaMalloc (their device memory is owned by another
@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2609_28568_b200 import binding as nb
 from paper_2609_28568_b200 import synth
 from parity import check_f32, f32
@@ -42,6 +43,22 @@ def test_no_alloc_matches_allocating_entry_point_twice_in_a_row():
             torch.cuda.synchronize()
             check_f32(got, f32(want).astype(np.float64), f"call {call}, accumulate={accumulate}")
             assert np.abs(f32(got)).max() > 0
+        # and on its own feet, against the oracle: the first call overwrote the 3.0 the buffer held
+        # with the column sums of dout * gelu'(pre), the second added the same sums again
+        dz = f32(dout).astype(np.float64) * oracle.gelu_grad(f32(pre).astype(np.float64))
+        check_f32(got, 2.0 * oracle.reduce_dbias(dz.astype(np.float32)), f"call {call} against the oracle")
+    # a call allocates nothing: free device memory is the same before and after a warmed-up call
+    BT, OC = 1024, 3072
+    dout = synth.normal(920, (BT, OC), 1e-3, dev)
+    pre = synth.normal(921, (BT, OC), 1.0, dev)
+    got = torch.zeros((OC,), dtype=torch.float32, device=dev)
+    nb.nb_gelu_dbias_noalloc(got, dout, pre, BT, OC, 0)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    nb.nb_gelu_dbias_noalloc(got, dout, pre, BT, OC, 1)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the allocation-free entry point changed the free device memory"
     # empty batch: accumulate=0 zeroes, accumulate=1 leaves the gradient alone
     g = torch.full((64,), 2.0, dtype=torch.float32, device=dev)
     nb.nb_gelu_dbias_noalloc(g, 16, 16, 0, 64, 1)

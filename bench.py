@@ -275,8 +275,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from the host in the timed region instead of replaying a CUDA graph")
-    ap.add_argument("--one-stream", action="store_true",
-                    help="keep the weight-gradient calls on the main stream (default: a second stream)")
+    ap.add_argument("--two-streams", action="store_true",
+                    help="issue the weight-gradient calls on a second stream, as separate launches (default: one "
+                         "stream, one launch per layer backward; the two arrangements time the same on a "
+                         "power-capped part)")
+    ap.add_argument("--one-stream", action="store_true", help="accepted for compatibility: this is the default")
     ap.add_argument("--dp", action="store_true",
                     help="data parallel instead of replicas: the same weights on every rank, its own rows, and "
                          "the fp32 gradients all-reduced (NCCL) in buckets under the last micro-step's backward; "
@@ -286,6 +289,11 @@ def main():
         args.no_graph = True
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started once, directly: start the N ranks here (one process per GPU); rank 0 prints the line
+        from paper_2609_28568_b200.launch import spawn_ranks
+        raise SystemExit(spawn_ranks(args.gpus, [os.path.abspath(__file__), *sys.argv[1:]]))
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -313,7 +321,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     model, BT, micro_steps, cfg_id, wgrad, wdesc = WORKLOADS[args.workload]
-    # weight gradients on a second stream (not with --dp: the reducer's events follow one stream)
+    # one stream in model order by default; --two-streams puts the weight gradients on a second one
     if model == "qwen3_lora":
         from paper_2609_28568_b200.stack import LoraStack
         if args.dp:
@@ -322,7 +330,7 @@ def main():
     else:
         stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
                             wgrad=wgrad, shared_weights=args.dp,
-                            wgrad_stream=not (args.dp or args.one_stream))
+                            wgrad_stream=bool(args.two_streams and not args.dp))
     reducer = None
     if args.dp:
         from paper_2609_28568_b200 import dp as dpmod
@@ -379,7 +387,7 @@ def main():
     sampler = ClockSampler(gpu_id)
     # One step is captured into a CUDA graph after the warm-up (every library call is
     # capturable: no allocation, no synchronisation) and the timed region replays it, so the
-    # 588 launches of a step cost the host one call.
+    # launches of a step (392 for the GPT-2 stack) cost the host one call.
     run_step, launches_per_step = stack.step, None
     if reducer is not None:
         run_step = lambda: stack.step_dp(reducer)  # noqa: E731
@@ -445,9 +453,9 @@ def main():
     # that is the "kernel timed inside a long step" case, compared with the sustained peak
     long_step = ms_per_step * (args.warmup + 2 * args.steps) > 1000.0
     peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
-    # Every launch of a step is an instantiation of the one GEMM kernel, so its average launch
-    # duration over the timed region is that region's length / launches, and algorithmic flops per
-    # launch / that duration is this rank's flops / time of the timed region. (The breakdown pass
+    # Every launch of a step is one of the two tensor-core GEMM kernels (forward; layer backward), so
+    # their average launch duration over the timed region is that region's length / launches, and
+    # algorithmic flops per launch / that duration is this rank's flops / time of the timed region. (The breakdown pass
     # below it has events between the calls, which cost it dependent-launch overlap: it is only
     # used for the per-call split.)
     my_ms_per_step = ev0.elapsed_time(ev1) / args.steps
@@ -464,9 +472,9 @@ def main():
         "bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
         "frac": achieved_tf / peak_tf, "traffic": traffic,
         "peak_source": f"{peak_src} cuBLAS bf16 ({'sustained' if long_step else 'burst'})",
-        "kernel": "nb::gemm_kernel (tcgen05 fwd / dgrad / wgrad instantiations): every launch of a step; "
-                  "average launch duration = timed region (CUDA events on the launch stream) / launches "
-                  "(with two streams the ends of launches overlap); "
+        "kernel": "nb::gemm_kernel (tcgen05 forward instantiations) and nb::layer_bwd_kernel (dinp tiles and "
+                  "dweight k-chunks of a layer in one launch): every launch of a step; "
+                  "average launch duration = timed region (CUDA events on the launch stream) / launches; "
                   "per_call from a second pass over the same steps with an event at every call boundary",
         "launches_per_step": launches / args.steps,
         "avg_launch_us": my_ms_per_step * 1e3 / (launches / args.steps) if launches else None,

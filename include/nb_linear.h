@@ -3,8 +3,8 @@
  *
  * The calls below are the part of a GPT-2 124M training step that takes most of its
  * time: the QKV, attention-output, MLP fc (+GELU), MLP projection and tied lm_head
- * products, forward and backward (paper: Results/Speed, the stage table: "GEMMs
- * (projections and head)"; layer shapes in Method/Model and Figure 1). The library
+ * products, forward and backward (paper: Results/Speed, the stage table, the row of
+ * the matrix products; layer shapes in Method/Model and Figure 1). The library
  * follows the paper's description of a C ABI that bindings in any language compose
  * from, with return codes that tell a malformed request from a failed execution
  * (paper: The stack under test).
@@ -27,9 +27,17 @@
  *    calling thread. NB_ERR_INVALID_ARG and NB_ERR_UNSUPPORTED are malformed requests
  *    and launch nothing. NB_ERR_CUDA is a driver / launch failure. NB_ERR_TIMEOUT is
  *    reported by nb_check_status when a kernel gave up on a bounded wait.
- *  - The library keeps a grow-only device workspace (only for backward calls that
- *    apply this layer's own activation derivative, see below), a 64-byte device status
- *    word per device and a host-side cache of TMA descriptors.
+ *  - The library keeps a grow-only device workspace, a 64-byte device status word per
+ *    device and a host-side cache of TMA descriptors. Two kinds of call use the
+ *    workspace: backward calls that apply this layer's own activation derivative
+ *    (act != NB_ACT_NONE: dz is formed there) and nb_lm_head_ce_forward (its softmax
+ *    partials). There is ONE workspace per device, so such calls must be ordered with
+ *    respect to each other: issue them on one stream, or order the streams with
+ *    events; two of them running at the same time overwrite each other's data. Growing
+ *    the workspace synchronises the device and frees the old one, which is not allowed
+ *    while a stream is being captured into a CUDA graph: size it first with
+ *    nb_workspace_reserve (a call that would have to grow it during a capture returns
+ *    NB_ERR_UNSUPPORTED and launches nothing).
  */
 #ifndef NB_LINEAR_H
 #define NB_LINEAR_H
@@ -72,7 +80,8 @@ int64_t nb_linear_out_elems(int64_t BT, int64_t OC, int act);
 
 /*
  * Forward: z = inp . weight^T (+ bias); out = act(z).
- * (paper: Figure 1, "768 -> 3072, GELU, 3072 -> 768"; head tied and bias-free)
+ * (paper: Figure 1, the MLP box of a block and the head box: the head is tied to the
+ * token embedding and has no bias)
  *
  *   out     [out] act == NONE : [BT, OC] bf16.
  *                 act != NONE : two planes back to back, the activated result first
@@ -153,9 +162,10 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
 int nb_reduce_dbias(void *dbias, const void *dout, int64_t BT, int64_t OC, int accumulate);
 
 /*
- * Head with fused cross-entropy statistics (paper: Figure 1, "cross-entropy over the first 50,257;
- * padding rows get no probability and no gradient", loss in f32; Results/Speed lists the
- * cross-entropy forward and backward as separate kernels next to the head's GEMMs).
+ * Head with fused cross-entropy statistics (paper: Figure 1, the loss box: the loss covers only
+ * the real vocabulary, the padding takes no part in it and receives no gradient, and it is
+ * computed in 32-bit; Results/Speed lists the cross-entropy forward and backward as separate
+ * kernels next to the head's GEMMs).
  *
  * nb_lm_head_ce_forward: logits = inp . weight^T (bf16, [BT, Vp], stored as by nb_linear_forward),
  * and, in the same pass, from the stored (rounded) logits of the first V columns:

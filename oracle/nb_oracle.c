@@ -132,11 +132,11 @@ int nbo_lora_forward_f64(double *out, const float *inp, const float *W, const fl
                          const float *A, const float *B, double scale, int64_t BT, int64_t C,
                          int64_t OC, int64_t r)
 {
-    if (!out || !inp || !W || !A || !B || BT < 0 || C <= 0 || OC <= 0 || r <= 0) return -1;
+    if (!out || !inp || !W || !A || !B || BT < 0 || C <= 0 || OC <= 0 || r <= 0 || r > 256) return -1;
 #pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < BT; ++m) {
         double t[256];
-        for (int64_t j = 0; j < r && j < 256; ++j) {
+        for (int64_t j = 0; j < r; ++j) {
             double acc = 0.0;
             for (int64_t k = 0; k < C; ++k) acc += (double)inp[m * C + k] * (double)A[j * C + k];
             t[j] = acc;
@@ -150,7 +150,7 @@ int nbo_lora_forward_f64(double *out, const float *inp, const float *W, const fl
             out[m * OC + o] = acc + scale * lo;
         }
     }
-    return r <= 256 ? 0 : -1;
+    return 0;
 }
 
 int nbo_lora_backward_f64(double *dinp, double *dA, double *dB, const float *dout, const float *inp,

@@ -381,9 +381,17 @@ int choose_splits(int tiles, int kblocks, int slots)
     return best;
 }
 
-int ensure_workspace(DeviceState &s, size_t bytes)
+int ensure_workspace(DeviceState &s, size_t bytes, cudaStream_t stream = nullptr)
 {
     if (s.workspace_bytes >= bytes) return NB_OK;
+    // growing synchronises the device and frees memory that kernels of a graph under
+    // construction may refer to: refuse instead of failing inside the runtime
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (stream != nullptr && cudaStreamIsCapturing(stream, &cs) != cudaSuccess) (void)cudaGetLastError();
+    if (cs != cudaStreamCaptureStatusNone)
+        return fail(NB_ERR_UNSUPPORTED,
+                    "the workspace would have to grow to %zu bytes during stream capture; call "
+                    "nb_workspace_reserve before capturing", bytes);
     if (s.workspace) {
         NB_CUDA(cudaDeviceSynchronize());
         NB_CUDA(cudaFree(s.workspace));
@@ -792,7 +800,7 @@ int nb_linear_backward_ex(void *dinp, void *dweight, void *dbias, const void *do
     // dz: either dout itself, or dout times this layer's activation derivative (workspace)
     const void *dz = dout;
     if (act != NB_ACT_NONE) {
-        if ((rc = ensure_workspace(*s, static_cast<size_t>(BT * OC) * 2)) != NB_OK) return rc;
+        if ((rc = ensure_workspace(*s, static_cast<size_t>(BT * OC) * 2, stream)) != NB_OK) return rc;
         if (act == NB_ACT_GELU) {
             const long long nvec = BT * OC / 8;
             gelu_backward_kernel<<<elementwise_grid(*s, nvec), 256, 0, stream>>>(
@@ -903,7 +911,7 @@ int nb_lm_head_ce_forward(void *logits, void *loss, void *lse, const void *inp, 
     DeviceState *s;
     if ((rc = get_state(&s)) != NB_OK) return rc;
     const int stats_ld = 2 * static_cast<int>((Vp + 255) / 256);
-    if ((rc = ensure_workspace(*s, static_cast<size_t>(BT) * stats_ld * sizeof(float2))) != NB_OK) return rc;
+    if ((rc = ensure_workspace(*s, static_cast<size_t>(BT) * stats_ld * sizeof(float2), stream)) != NB_OK) return rc;
     GemmArgs a;
     memset(&a, 0, sizeof(a));
     a.A = inp; a.a_rows = BT; a.a_cols = C;

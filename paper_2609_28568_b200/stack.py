@@ -295,6 +295,12 @@ class LinearStack:
 
         for ms in range(self.micro_steps):
             self.forward(ms, hook)
+            if ms == last:
+                # The last backward runs on the current stream alone (it has a hook), and the
+                # reducer's events are recorded there. Earlier micro-steps may have left weight-
+                # gradient kernels on the second stream: they must have accumulated before this
+                # micro-step adds to the same buffers and before a bucket is reduced.
+                self.join()
             self.backward(ms, on_call if ms == last else hook)
         reducer.finish()
 

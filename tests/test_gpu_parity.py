@@ -572,6 +572,26 @@ def test_flat_gradient_buckets_give_the_same_gradients_on_one_rank():
         assert rel_frob(f32(Lb.dbias), f32(La.dbias)) < 1e-5
 
 
+def test_data_parallel_step_with_the_second_stream_orders_its_accumulations():
+    """`step_dp` on a stack that issues weight gradients on a second stream: the micro-steps before
+    the last leave accumulations on that stream, the last one (and the reducer's events) runs on the
+    current stream. The gradients must equal those of the plain step."""
+    from paper_2609_28568_b200 import dp
+    from paper_2609_28568_b200.stack import LinearStack
+    a = LinearStack("gpt2_block", BT=2048, micro_steps=4, device=DEV, config_id=2)
+    a.step()
+    b = LinearStack("gpt2_block", BT=2048, micro_steps=4, device=DEV, config_id=2, wgrad_stream=True)
+    gb = b.attach_gradient_buckets(bucket_bytes=4 << 20)
+    red = dp.GradAllReducer(gb, None)
+    for _ in range(3):
+        b.step_dp(red)
+    torch.cuda.synchronize()
+    for La, Lb in zip(a.layers, b.layers):
+        assert rel_frob(f32(Lb.dweight), f32(La.dweight)) < 1e-5, La.spec.name
+        assert rel_frob(f32(Lb.dbias), f32(La.dbias)) < 1e-5, La.spec.name
+        assert torch.equal(Lb.dinp, La.dinp), La.spec.name
+
+
 @pytest.mark.parametrize("act", [nb.ACT_NONE, nb.ACT_GELU])
 def test_bias_reaches_every_tile_full_tensor(act):
     """Every element of a many-tile result carries ITS column's bias: the result with a large bias

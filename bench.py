@@ -455,9 +455,9 @@ def main():
     peak_tf = peaks["bf16_tflops_sustained"] if long_step else peaks["bf16_tflops"]
     # Every launch of a step is one of the two tensor-core GEMM kernels (forward; layer backward), so
     # their average launch duration over the timed region is that region's length / launches, and
-    # algorithmic flops per launch / that duration is this rank's flops / time of the timed region. (The breakdown pass
-    # below it has events between the calls, which cost it dependent-launch overlap: it is only
-    # used for the per-call split.)
+    # algorithmic flops per launch / that duration is this rank's flops / time of the timed region.
+    # (The breakdown pass below it has events between the calls, which cost it dependent-launch
+    # overlap: it is only used for the per-call split.)
     my_ms_per_step = ev0.elapsed_time(ev1) / args.steps
     achieved_tf = flops_step / (my_ms_per_step * 1e-3) / 1e12
     breakdown_tf = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0

@@ -313,6 +313,20 @@ int nb_debug_layer_bwd_plan(int64_t BT, int64_t C, int64_t OC, int pairs, int ge
  */
 int nb_debug_wait_timeout(int64_t limit_us);
 
+/*
+ * Self-test of the GEMM kernel's own time-out exit (paper: The stack under test asks of the
+ * surface that a failed execution is told apart from a malformed request; this is how the
+ * former is exercised without a fault): a one-tile, one-CTA forward product
+ * out[128, 256] = inp[128, 256] . weight[256, 256]^T in which the producer warp stops after two
+ * of the four k-blocks. The MMA issuer's bounded wait for the third stage runs out after
+ * `limit_us` microseconds (100 .. 1000000), it records the event in the device status word, the
+ * other roles see the abort flag, and every thread leaves through the kernel's common exit
+ * (wait for copies in flight, free tensor memory). `out` is left unwritten. Afterwards
+ * nb_check_status() reports NB_ERR_TIMEOUT naming wait 300 + stage; the context stays usable.
+ * All three pointers are device pointers, 16-byte aligned, bf16, dense row-major.
+ */
+int nb_debug_gemm_timeout(void *out, const void *inp, const void *weight, int64_t limit_us);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,7 @@ EXPORTS = (
     "nb_reduce_dbias", "nb_workspace_reserve", "nb_release", "nb_check_status",
     "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
     "nb_debug_split_plan", "nb_cast_f32_to_bf16", "nb_lm_head_ce_forward", "nb_ce_backward",
-    "nb_lora_linear_forward", "nb_lora_linear_backward", "nb_debug_layer_bwd_plan",
+    "nb_lora_linear_forward", "nb_lora_linear_backward", "nb_debug_layer_bwd_plan", "nb_debug_gemm_timeout",
 )
 
 _lib = None
@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         L.nb_lm_head_ce_forward.argtypes = [_vp] * 6 + [_i64] * 4 + [_vp]
         L.nb_ce_backward.argtypes = [_vp] * 4 + [ctypes.c_float] + [_i64] * 3 + [_vp]
         L.nb_debug_split_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int)]
+        L.nb_debug_gemm_timeout.argtypes = [_vp, _vp, _vp, _i64]
         L.nb_debug_layer_bwd_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int), _i64]
         _lib = L
     return _lib
@@ -215,6 +216,12 @@ def nb_debug_layer_bwd_plan(BT: int, C: int, OC: int, pairs: int, gelu_grad: boo
 
 def nb_kernel_launches() -> int:
     return int(lib().nb_kernel_launches())
+
+
+def nb_debug_gemm_timeout(out, inp, weight, limit_us: int) -> None:
+    """One-tile forward GEMM whose producer stops half way: exercises the kernel's time-out exit."""
+    lib().nb_set_stream(_stream())
+    _check(lib().nb_debug_gemm_timeout(_ptr(out), _ptr(inp), _ptr(weight), limit_us))
 
 
 def nb_debug_wait_timeout(limit_us: int) -> None:

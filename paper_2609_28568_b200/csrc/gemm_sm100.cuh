@@ -68,6 +68,8 @@ struct GemmParams {
     int v_real;                 //   columns >= v_real take no part in the statistics
     int *status;
     unsigned long long timeout_ns;
+    int debug_stop_kb;  // self-test of the time-out exit: the producer stops before this k-block
+                        // (counted over the CTA's whole run); negative in normal use
 };
 
 template <int CG_, int BLOCK_N_, int STAGES_, int NSTG_, bool A_MN_, bool B_MN_, int EPI_,
@@ -337,6 +339,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t tmem_base = ptx::ld_shared_u32_volatile(tmem_slot);
 
     const WaitCtx wctx{abort_addr, p.status, p.timeout_ns};
+    // The epilogue waits for a whole unit where the issuer waits for one stage: with twice the limit
+    // the wait that is closest to the cause of a stall is the one that expires and gets reported.
+    const WaitCtx wctx_epi{abort_addr, p.status, 2 * p.timeout_ns};
     const int num_units = p.tiles_m * p.tiles_n * p.splits;
 
     // one tile load, counted on the leader CTA's barrier
@@ -355,6 +360,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            int issued = 0;  // k-blocks loaded so far
             for (int u = first_unit; u < num_units && ok; u += unit_stride) {
                 int m_blk, n_blk, split;
                 decode_unit(p, u, m_blk, n_blk, split);
@@ -363,6 +369,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const int m0 = m_blk * Cfg::TILE_M + static_cast<int>(rank) * kBlockM;
                 const int kb_end = kb1 + p.kblocks_ext;  // the adapter term's k-blocks come last
                 for (int kb = kb0; kb < kb_end; ++kb) {
+                    // self-test only: leave the rest unloaded, so that the issuer's wait for this
+                    // stage runs out and the kernel leaves through its time-out exit
+                    if (issued++ == p.debug_stop_kb) {
+                        ok = false;
+                        break;
+                    }
                     const bool ext = kb >= kb1;
                     const CUtensorMap *mapA = ext ? &tmA2 : &tmA;
                     const CUtensorMap *mapB = ext ? &tmB2 : &tmB;
@@ -610,7 +622,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 }
             }
             bool ok = true;
-            if (lane == 0) ok = wait_barrier(wctx, tfull_bar(acc), acc_phase, 400 + acc);
+            if (lane == 0) ok = wait_barrier(wctx_epi, tfull_bar(acc), acc_phase, 400 + acc);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
             ptx::tc_fence_after();
@@ -704,7 +716,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     if (EPI == kEpiMulGeluGrad) {
                         bool aok = true;
                         if (lane == 0)
-                            aok = wait_barrier(wctx, waux_bar(g & 1u), (g >> 1) & 1u, 500 + ew);
+                            aok = wait_barrier(wctx_epi, waux_bar(g & 1u), (g >> 1) & 1u, 500 + ew);
                         aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
                         if (!aok) {
                             ptx::st_shared_u32_volatile(epi_abort_addr, 1);
@@ -863,7 +875,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ptx::named_bar_sync(1, kEpiThreads);
 
             bool ok = true;
-            if (lane == 0) ok = wait_barrier(wctx, tfull_bar(acc), acc_phase, 400 + acc);
+            if (lane == 0) ok = wait_barrier(wctx_epi, tfull_bar(acc), acc_phase, 400 + acc);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
             ptx::tc_fence_after();

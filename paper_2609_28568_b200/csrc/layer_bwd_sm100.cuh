@@ -254,6 +254,9 @@ layer_bwd_kernel(const __grid_constant__ CUtensorMap tmDz,    // dz   [BT, OC] b
     ptx::grid_dependency_wait();
     const uint32_t tmem_base = ptx::ld_shared_u32_volatile(tmem_slot);
     const WaitCtx wctx{abort_addr, p.status, p.timeout_ns};
+    // The epilogue waits for a whole unit where the issuer waits for one stage: with twice the limit
+    // the wait that is closest to the cause of a stall is the one that expires and gets reported.
+    const WaitCtx wctx_epi{abort_addr, p.status, 2 * p.timeout_ns};
 
     if (warp < 4) {
         ptx::setmaxnreg_dec<56>();
@@ -474,7 +477,7 @@ layer_bwd_kernel(const __grid_constant__ CUtensorMap tmDz,    // dz   [BT, OC] b
                 const int m0 = u.m_blk * 256 + static_cast<int>(rank) * 128;
                 const int nw = u.n_blk * 256 + hf * 128;  // this warp's first column
                 bool ok = true;
-                if (lane == 0) ok = wait_barrier(wctx, tfull_bar(acc), acc_phase, 400 + acc);
+                if (lane == 0) ok = wait_barrier(wctx_epi, tfull_bar(acc), acc_phase, 400 + acc);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) ptx::st_shared_u32_volatile(epi_abort_addr, 1);
                 ptx::tc_fence_after();
@@ -529,7 +532,7 @@ layer_bwd_kernel(const __grid_constant__ CUtensorMap tmDz,    // dz   [BT, OC] b
                             __syncwarp();
                             if (GELU_GRAD) {
                                 bool aok = true;
-                                if (lane == 0) aok = wait_barrier(wctx, waux_bar(g & 1u), (g >> 1) & 1u, 500 + ew);
+                                if (lane == 0) aok = wait_barrier(wctx_epi, waux_bar(g & 1u), (g >> 1) & 1u, 500 + ew);
                                 aok = __shfl_sync(0xffffffffu, aok ? 1 : 0, 0) != 0;
                                 if (!aok) {
                                     ptx::st_shared_u32_volatile(epi_abort_addr, 1);

@@ -206,6 +206,8 @@ struct GemmArgs {
     float2 *stats; // forward with softmax statistics: [M, stats_ld]
     int stats_ld;
     int v_real;
+    int debug_stop_kb;                  // nb_debug_gemm_timeout only: see GemmParams; 0 = unset (-1 is passed on)
+    unsigned long long debug_timeout_ns;  //   and its shortened wait limit
 };
 
 template <class Cfg>
@@ -282,7 +284,8 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     p.stats_ld = a.stats_ld;
     p.v_real = a.v_real;
     p.status = s.status;
-    p.timeout_ns = kDefaultTimeoutNs;
+    p.timeout_ns = a.debug_timeout_ns ? a.debug_timeout_ns : kDefaultTimeoutNs;
+    p.debug_stop_kb = a.debug_stop_kb > 0 ? a.debug_stop_kb : -1;
     const long long units = 1ll * p.tiles_m * p.tiles_n * p.splits;
     if (units <= 0 || units >= (1ll << 31)) return fail(NB_ERR_UNSUPPORTED, "tile count out of range");
     const int clusters = static_cast<int>(units < max_clusters[dev] ? units : max_clusters[dev]);
@@ -1153,6 +1156,30 @@ int nb_debug_layer_bwd_plan(int64_t BT, int64_t C, int64_t OC, int pairs, int ge
         }
     }
     return records;
+}
+
+int nb_debug_gemm_timeout(void *out, const void *inp, const void *weight, int64_t limit_us)
+{
+    if (!out || !inp || !weight) return fail(NB_ERR_INVALID_ARG, "out, inp and weight must not be NULL");
+    if (!aligned16(out) || !aligned16(inp) || !aligned16(weight))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (limit_us < 100 || limit_us > 1000000)
+        return fail(NB_ERR_INVALID_ARG, "limit_us must be within [100, 1000000]");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    int rc = get_state(&s);
+    if (rc != NB_OK) return rc;
+    const int64_t BT = 128, C = 256, OC = 256;  // one tile, one CTA, four k-blocks
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = weight; a.b_rows = OC; a.b_cols = C;
+    a.D = out; a.d_rows = BT; a.d_cols = OC; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(OC); a.K = static_cast<int>(C);
+    a.splits = 1;
+    a.debug_stop_kb = 2;  // the first two k-blocks are loaded, the third never is
+    a.debug_timeout_ns = static_cast<unsigned long long>(limit_us) * 1000ull;
+    return launch_gemm<FwdStore1>(*s, a, g_stream);
 }
 
 int nb_debug_wait_timeout(int64_t limit_us)

@@ -263,6 +263,26 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     run_layer_full(128, 64, 256, nb.ACT_NONE, seed=61)
 
 
+def test_gemm_kernel_time_out_exit_and_recovery():
+    """The GEMM kernel's own abort path: a producer that stops half way makes the issuer's bounded
+    wait expire; the kernel must return by itself (no trap, no fault), report which wait gave up,
+    leave the canaries around its output alone, and the next call on the same context must be right."""
+    inp, w = gen(91, (128, 256), 1.0), gen(92, (256, 256), 0.02)
+    out = Guarded((128, 256), torch.bfloat16)
+    nb.nb_debug_gemm_timeout(out.t, inp, w, 3000)
+    with pytest.raises(nb.NbError) as e:
+        nb.nb_check_status()
+    assert e.value.code == nb.NB_ERR_TIMEOUT
+    assert "wait id 302" in str(e.value)  # the issuer's wait for the third stage
+    out.check("aborted GEMM")
+    nb.nb_check_status()  # cleared
+    nb.nb_linear_forward_ex(out.t, None, inp, w, None, 128, 256, 256, nb.ACT_NONE)
+    o_ref, _ = oracle.linear_forward(f32(inp), f32(w))
+    check_bf16(out.t, o_ref, "the same product after the aborted one")
+    out.check("after recovery")
+    run_layer_full(392, 328, 528, nb.ACT_GELU, seed=93)
+
+
 def test_other_stream():
     s = torch.cuda.Stream()
     BT, C, OC = 512, 256, 512

@@ -217,6 +217,44 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
                             int64_t OC, int64_t r, int accumulate, void *stream);
 
 /*
+ * Adapters that share an input, stacked (paper: Method/The clinical stage: the query, key and value
+ * projections of a layer read the same activations, and so do the gate and up projections; each of
+ * the seven projections has its own rank-16 adapter). Stacking the A matrices of such a group row
+ * by row gives one rank-R product for the whole group instead of one skinny product per adapter,
+ * and the input is read once:
+ *
+ *   nb_lora_down_stacked:            t_stack = bf16( scale * inp . a_stack^T )   [BT, R]
+ *                                    a_stack [R, C] = the groups' A matrices one after the other
+ *   nb_lora_linear_forward_stacked:  out = inp . weight^T (+ bias) + t_stack[:, off:off+r] . lora_b^T
+ *                                    (one GEMM, as in nb_lora_linear_forward; t_stack is an input)
+ *   nb_lora_linear_backward_stacked: u_stack[:, off:off+r] = bf16( scale * dout . lora_b )
+ *                                    dinp    = dout . weight + u_stack[:, off:off+r] . lora_a
+ *                                    dlora_b (+)= dout^T . t_stack[:, off:off+r]       [OC, r] fp32
+ *                                    (lora_a [r, C] is this adapter's rows of a_stack; dinp and dlora_b
+ *                                    may be NULL; the gradient of A is NOT formed here)
+ *   nb_lora_da_stacked:              da_stack (+)= u_stack^T . inp                    [R, C] fp32
+ *                                    once per group, after the backward calls of all its members have
+ *                                    filled their columns of u_stack; rows [off, off+r) are that
+ *                                    adapter's dlora_a
+ *
+ * r and off are multiples of 8, off + r <= R <= 64, R a multiple of 8. Column slices of t_stack and
+ * u_stack are addressed in place (row stride R); columns outside a slice are neither read into a
+ * product nor written. Every result equals what the unstacked calls give for that adapter; rounding
+ * points and all other conventions are those of nb_lora_linear_forward / _backward.
+ */
+int nb_lora_down_stacked(void *t_stack, const void *inp, const void *a_stack, float scale, int64_t BT,
+                         int64_t C, int64_t R, void *stream);
+int nb_lora_linear_forward_stacked(void *out, const void *inp, const void *weight, const void *bias,
+                                   const void *t_stack, const void *lora_b, int64_t BT, int64_t C,
+                                   int64_t OC, int64_t r, int64_t R, int64_t off, void *stream);
+int nb_lora_linear_backward_stacked(void *dinp, void *dlora_b, void *u_stack, const void *dout,
+                                    const void *weight, const void *lora_a, const void *lora_b,
+                                    const void *t_stack, float scale, int64_t BT, int64_t C, int64_t OC,
+                                    int64_t r, int64_t R, int64_t off, int accumulate, void *stream);
+int nb_lora_da_stacked(void *da_stack, const void *u_stack, const void *inp, int64_t BT, int64_t C,
+                       int64_t R, int accumulate, void *stream);
+
+/*
  * Master-weight cast: dst[i] = bf16(src[i]), round to nearest even, for n elements.
  * (paper: Method/Optimisation and precision keeps fp32 master weights and bf16 compute copies;
  * Results/Speed, the table of levers: the cast is done once per optimizer step and reused by

@@ -25,6 +25,8 @@ EXPORTS = (
     "nb_debug_wait_timeout", "nb_kernel_launches", "nb_gelu_dbias_noalloc",
     "nb_debug_split_plan", "nb_cast_f32_to_bf16", "nb_lm_head_ce_forward", "nb_ce_backward",
     "nb_lora_linear_forward", "nb_lora_linear_backward", "nb_debug_layer_bwd_plan", "nb_debug_gemm_timeout",
+    "nb_lora_down_stacked", "nb_lora_linear_forward_stacked", "nb_lora_linear_backward_stacked",
+    "nb_lora_da_stacked",
 )
 
 _lib = None
@@ -64,6 +66,10 @@ def lib() -> ctypes.CDLL:
         L.nb_cast_f32_to_bf16.argtypes = [_vp, _vp, _i64, _vp]
         L.nb_lora_linear_forward.argtypes = [_vp] * 7 + [ctypes.c_float] + [_i64] * 4 + [_vp]
         L.nb_lora_linear_backward.argtypes = [_vp] * 10 + [ctypes.c_float] + [_i64] * 4 + [_int, _vp]
+        L.nb_lora_down_stacked.argtypes = [_vp, _vp, _vp, ctypes.c_float, _i64, _i64, _i64, _vp]
+        L.nb_lora_linear_forward_stacked.argtypes = [_vp] * 6 + [_i64] * 6 + [_vp]
+        L.nb_lora_linear_backward_stacked.argtypes = [_vp] * 8 + [ctypes.c_float] + [_i64] * 6 + [_int, _vp]
+        L.nb_lora_da_stacked.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64, _int, _vp]
         L.nb_lm_head_ce_forward.argtypes = [_vp] * 6 + [_i64] * 4 + [_vp]
         L.nb_ce_backward.argtypes = [_vp] * 4 + [ctypes.c_float] + [_i64] * 3 + [_vp]
         L.nb_debug_split_plan.argtypes = [_i64, _i64, _i64, _int, _int, ctypes.POINTER(_int)]
@@ -174,6 +180,35 @@ def nb_lora_linear_backward(dinp, dlora_a, dlora_b, u, dout, inp, weight, lora_a
                                          _ptr(inp), _ptr(weight), _ptr(lora_a), _ptr(lora_b), _ptr(t),
                                          scale, BT, C, OC, r, int(accumulate),
                                          _stream() if stream is None else stream))
+
+
+def nb_lora_down_stacked(t_stack, inp, a_stack, scale, BT, C, R, stream=None) -> None:
+    """t_stack = bf16(scale * inp @ a_stack.T): the down-projections of all adapters of a group at once."""
+    _check(lib().nb_lora_down_stacked(_ptr(t_stack), _ptr(inp), _ptr(a_stack), scale, BT, C, R,
+                                      _stream() if stream is None else stream))
+
+
+def nb_lora_linear_forward_stacked(out, inp, weight, bias, t_stack, lora_b, BT, C, OC, r, R, off,
+                                   stream=None) -> None:
+    """out = inp @ W.T (+ bias) + t_stack[:, off:off+r] @ B.T, the adapter term fused in."""
+    _check(lib().nb_lora_linear_forward_stacked(_ptr(out), _ptr(inp), _ptr(weight), _ptr(bias), _ptr(t_stack),
+                                                _ptr(lora_b), BT, C, OC, r, R, off,
+                                                _stream() if stream is None else stream))
+
+
+def nb_lora_linear_backward_stacked(dinp, dlora_b, u_stack, dout, weight, lora_a, lora_b, t_stack, scale, BT, C,
+                                    OC, r, R, off, accumulate, stream=None) -> None:
+    """u slice, dinp and dB of one adapted projection of a stacked group (dA comes from nb_lora_da_stacked)."""
+    _check(lib().nb_lora_linear_backward_stacked(_ptr(dinp), _ptr(dlora_b), _ptr(u_stack), _ptr(dout),
+                                                 _ptr(weight), _ptr(lora_a), _ptr(lora_b), _ptr(t_stack), scale,
+                                                 BT, C, OC, r, R, off, int(accumulate),
+                                                 _stream() if stream is None else stream))
+
+
+def nb_lora_da_stacked(da_stack, u_stack, inp, BT, C, R, accumulate, stream=None) -> None:
+    """da_stack (+)= u_stack.T @ inp: the A gradients of all adapters of a group at once."""
+    _check(lib().nb_lora_da_stacked(_ptr(da_stack), _ptr(u_stack), _ptr(inp), BT, C, R, int(accumulate),
+                                    _stream() if stream is None else stream))
 
 
 def nb_lm_head_ce_forward(logits, loss, lse, inp, weight, targets, BT, C, Vp, V, stream=None) -> None:

@@ -54,11 +54,11 @@ int fail(int code, const char *fmt, ...)
 // ----------------------------------------------------------------------------- per-device state
 struct TmapKey {
     const void *ptr;
-    uint64_t rows, cols;
+    uint64_t rows, cols, ld;
     uint32_t box_cols, box_rows, dtype;
     bool operator==(const TmapKey &o) const
     {
-        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_cols == o.box_cols &&
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_cols == o.box_cols &&
                box_rows == o.box_rows && dtype == o.dtype;
     }
 };
@@ -68,6 +68,7 @@ struct TmapKeyHash {
         uint64_t h = reinterpret_cast<uint64_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
         h ^= (k.rows + 0x7F4A7C15ull) * 0xBF58476D1CE4E5B9ull;
         h ^= (k.cols + 0x165667B1ull) * 0x94D049BB133111EBull;
+        h ^= (k.ld + 0x2545F491ull) * 0xD6E8FEB86659FD93ull;
         h ^= (static_cast<uint64_t>(k.box_cols) << 40) ^ (static_cast<uint64_t>(k.box_rows) << 20) ^
              k.dtype;
         return static_cast<size_t>(h ^ (h >> 29));
@@ -124,19 +125,25 @@ int get_state(DeviceState **out)
 
 // Row-major [rows, cols] tensor, tiles of box_rows x box_cols with the 128-byte swizzle.
 // dtype: 0 bf16, 1 fp32. The innermost box extent is always 128 bytes (64 bf16 / 32 fp32).
+// ld: elements from one row to the next (0: dense, = cols); a column slice of a wider tensor is a
+// view with ld > cols, and what lies beyond its cols reads as zero and is never written.
 int get_tmap(DeviceState &s, CUtensorMap *out, const void *ptr, uint64_t rows, uint64_t cols,
-             uint32_t dtype, uint32_t box_rows)
+             uint32_t dtype, uint32_t box_rows, uint64_t ld = 0)
 {
     const uint32_t esz = dtype == 0 ? 2u : 4u;
     const uint32_t box_cols = 128u / esz;
-    TmapKey key{ptr, rows, cols, box_cols, box_rows, dtype};
+    if (ld == 0) ld = cols;
+    if (ld < cols || (ld * esz) % 16 != 0)
+        return fail(NB_ERR_UNSUPPORTED, "row stride of %llu elements is not a multiple of 16 bytes",
+                    static_cast<unsigned long long>(ld));
+    TmapKey key{ptr, rows, cols, ld, box_cols, box_rows, dtype};
     auto it = s.tmaps.find(key);
     if (it != s.tmaps.end()) {
         *out = it->second;
         return NB_OK;
     }
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * esz};
+    cuuint64_t strides[1] = {ld * esz};
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     // The encoder does not write every byte of the opaque descriptor: start from zeros, otherwise
@@ -203,6 +210,7 @@ struct GemmArgs {
     const void *B2; uint64_t b2_rows, b2_cols;
     int k2;
     float alpha;   // D = alpha * acc (+ bias); 0 is read as 1
+    uint64_t a_ld, b_ld, d_ld, a2_ld;  // row strides in elements of A, B, D, A2 when they are column slices (0: dense)
     float2 *stats; // forward with softmax statistics: [M, stats_ld]
     int stats_ld;
     int v_real;
@@ -243,9 +251,9 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     CUtensorMap tA, tB, tD, tE;
     int rc;
     // operands are fetched as 64 x 64 boxes; results (and the aux tile) move as 128-row chunks
-    if ((rc = get_tmap(s, &tA, a.A, a.a_rows, a.a_cols, 0, 64)) != NB_OK) return rc;
-    if ((rc = get_tmap(s, &tB, a.B, a.b_rows, a.b_cols, 0, 64)) != NB_OK) return rc;
-    if ((rc = get_tmap(s, &tD, a.D, a.d_rows, a.d_cols, a.d_dtype, Cfg::OUT_BOX_ROWS)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tA, a.A, a.a_rows, a.a_cols, 0, 64, a.a_ld)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tB, a.B, a.b_rows, a.b_cols, 0, 64, a.b_ld)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tD, a.D, a.d_rows, a.d_cols, a.d_dtype, Cfg::OUT_BOX_ROWS, a.d_ld)) != NB_OK) return rc;
     if (a.E) {
         if ((rc = get_tmap(s, &tE, a.E, a.e_rows, a.e_cols, 0, Cfg::OUT_BOX_ROWS)) != NB_OK) return rc;
     } else {
@@ -253,7 +261,7 @@ int launch_gemm(DeviceState &s, const GemmArgs &a, cudaStream_t stream)
     }
     CUtensorMap tA2 = tA, tB2 = tB;
     if (a.A2 && a.B2 && a.k2 > 0) {
-        if ((rc = get_tmap(s, &tA2, a.A2, a.a2_rows, a.a2_cols, 0, 64)) != NB_OK) return rc;
+        if ((rc = get_tmap(s, &tA2, a.A2, a.a2_rows, a.a2_cols, 0, 64, a.a2_ld)) != NB_OK) return rc;
         if ((rc = get_tmap(s, &tB2, a.B2, a.b2_rows, a.b2_cols, 0, 64)) != NB_OK) return rc;
     }
     GemmParams p;
@@ -440,12 +448,13 @@ int elementwise_grid(const DeviceState &s, long long nvec)
 // dweight[M_, N_] (+)= dz^T . inp over BT rows, fp32, with the split-K factor chosen per shape;
 // dz [BT, M_], inp [BT, N_]. dbias (or null) is summed inside the same kernel.
 int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight, float *dbias,
-                  int64_t BT, int64_t M_, int64_t N_, int accumulate, cudaStream_t stream)
+                  int64_t BT, int64_t M_, int64_t N_, int accumulate, cudaStream_t stream,
+                  uint64_t inp_ld = 0)
 {
     GemmArgs a;
     memset(&a, 0, sizeof(a));
     a.A = dz; a.a_rows = BT; a.a_cols = M_;
-    a.B = inp; a.b_rows = BT; a.b_cols = N_;
+    a.B = inp; a.b_rows = BT; a.b_cols = N_; a.b_ld = inp_ld;
     a.D = dweight; a.d_rows = M_; a.d_cols = N_; a.d_dtype = 1;
     a.M = static_cast<int>(M_); a.N = static_cast<int>(N_); a.K = static_cast<int>(BT);
     const bool narrow = dbias == nullptr && a.N <= kNarrowN;
@@ -1051,6 +1060,147 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
         if ((rc = run_wgrad_f32(*s, u, inp, dlora_a, nullptr, BT, r, C, accumulate, stream)) != NB_OK)
             return rc;
     return NB_OK;
+}
+
+// --- adapters that share an input, stacked (q, k, v; gate, up): one rank-R product for all of them
+namespace {
+int check_stack(int64_t r, int64_t R, int64_t off)
+{
+    if (r < 8 || r > 64 || r % 8 != 0) return fail(NB_ERR_UNSUPPORTED, "rank must be 8..64, a multiple of 8");
+    if (R < r || R > 64 || R % 8 != 0)
+        return fail(NB_ERR_UNSUPPORTED, "stacked rank must be a multiple of 8, at least r and at most 64");
+    if (off < 0 || off % 8 != 0 || off + r > R)
+        return fail(NB_ERR_INVALID_ARG, "slice [%lld, %lld) does not lie in the %lld stacked columns",
+                    static_cast<long long>(off), static_cast<long long>(off + r), static_cast<long long>(R));
+    return NB_OK;
+}
+}  // namespace
+
+int nb_lora_down_stacked(void *t_stack, const void *inp, const void *a_stack, float scale, int64_t BT,
+                         int64_t C, int64_t R, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, R);
+    if (rc != NB_OK) return rc;
+    if (R > 64) return fail(NB_ERR_UNSUPPORTED, "stacked rank must be at most 64");
+    if (!t_stack || !inp || !a_stack) return fail(NB_ERR_INVALID_ARG, "t_stack, inp and a_stack must not be NULL");
+    if (!aligned16(t_stack) || !aligned16(inp) || !aligned16(a_stack))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (BT == 0) return NB_OK;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));  // t_stack = scale * inp . a_stack^T
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = a_stack; a.b_rows = R; a.b_cols = C;
+    a.D = t_stack; a.d_rows = BT; a.d_cols = R; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(R); a.K = static_cast<int>(C);
+    a.splits = 1;
+    a.alpha = scale;
+    return launch_gemm<FwdStoreNarrow>(*s, a, stream);
+}
+
+int nb_lora_linear_forward_stacked(void *out, const void *inp, const void *weight, const void *bias,
+                                   const void *t_stack, const void *lora_b, int64_t BT, int64_t C,
+                                   int64_t OC, int64_t r, int64_t R, int64_t off, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, OC);
+    if (rc != NB_OK) return rc;
+    if ((rc = check_stack(r, R, off)) != NB_OK) return rc;
+    if (!out || !inp || !weight || !t_stack || !lora_b)
+        return fail(NB_ERR_INVALID_ARG, "out, inp, weight, t_stack and lora_b must not be NULL");
+    if (!aligned16(out) || !aligned16(inp) || !aligned16(weight) || !aligned16(t_stack) || !aligned16(lora_b))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (BT == 0) return NB_OK;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));  // out = inp . W^T (+ bias) + t_slice . B^T: r extra columns of K
+    a.A = inp; a.a_rows = BT; a.a_cols = C;
+    a.B = weight; a.b_rows = OC; a.b_cols = C;
+    a.D = out; a.d_rows = BT; a.d_cols = OC; a.d_dtype = 0;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(OC); a.K = static_cast<int>(C);
+    a.bias = bias;
+    a.splits = 1;
+    a.A2 = static_cast<const uint16_t *>(t_stack) + off; a.a2_rows = BT; a.a2_cols = r; a.a2_ld = R;
+    a.B2 = lora_b; a.b2_rows = OC; a.b2_cols = r;
+    a.k2 = static_cast<int>(r);
+    return launch_gemm_auto<FwdStore1, FwdStore2>(*s, a, stream);
+}
+
+int nb_lora_linear_backward_stacked(void *dinp, void *dlora_b, void *u_stack, const void *dout,
+                                    const void *weight, const void *lora_a, const void *lora_b,
+                                    const void *t_stack, float scale, int64_t BT, int64_t C, int64_t OC,
+                                    int64_t r, int64_t R, int64_t off, int accumulate, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, OC);
+    if (rc != NB_OK) return rc;
+    if ((rc = check_stack(r, R, off)) != NB_OK) return rc;
+    if (!u_stack || !dout || !lora_a || !lora_b)
+        return fail(NB_ERR_INVALID_ARG, "u_stack, dout, lora_a and lora_b must not be NULL");
+    if (dinp && !weight) return fail(NB_ERR_INVALID_ARG, "weight is required to compute dinp");
+    if (dlora_b && !t_stack) return fail(NB_ERR_INVALID_ARG, "t_stack (from the forward calls) is required for dlora_b");
+    if (!aligned16(dinp) || !aligned16(dlora_b) || !aligned16(u_stack) || !aligned16(dout) || !aligned16(weight) ||
+        !aligned16(lora_a) || !aligned16(lora_b) || !aligned16(t_stack))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    if (BT == 0) {
+        if (!accumulate && dlora_b) NB_CUDA(cudaMemsetAsync(dlora_b, 0, static_cast<size_t>(OC * r) * 4, stream));
+        return NB_OK;
+    }
+    uint16_t *u_slice = static_cast<uint16_t *>(u_stack) + off;
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));  // u_slice = scale * dout . B
+    a.A = dout; a.a_rows = BT; a.a_cols = OC;
+    a.B = lora_b; a.b_rows = OC; a.b_cols = r;
+    a.D = u_slice; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0; a.d_ld = R;
+    a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
+    a.splits = 1;
+    a.alpha = scale;
+    if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    if (dinp) {  // dinp = dout . W + u_slice . A
+        memset(&a, 0, sizeof(a));
+        a.A = dout; a.a_rows = BT; a.a_cols = OC;
+        a.B = weight; a.b_rows = OC; a.b_cols = C;
+        a.D = dinp; a.d_rows = BT; a.d_cols = C; a.d_dtype = 0;
+        a.M = static_cast<int>(BT); a.N = static_cast<int>(C); a.K = static_cast<int>(OC);
+        a.splits = 1;
+        a.A2 = u_slice; a.a2_rows = BT; a.a2_cols = r; a.a2_ld = R;
+        a.B2 = lora_a; a.b2_rows = r; a.b2_cols = C;
+        a.k2 = static_cast<int>(r);
+        if ((rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream)) != NB_OK) return rc;
+    }
+    if (dlora_b)  // dB [OC, r] (+)= dout^T . t_slice
+        if ((rc = run_wgrad_f32(*s, dout, static_cast<const uint16_t *>(t_stack) + off, dlora_b, nullptr, BT, OC, r,
+                                accumulate, stream, static_cast<uint64_t>(R))) != NB_OK)
+            return rc;
+    return NB_OK;
+}
+
+int nb_lora_da_stacked(void *da_stack, const void *u_stack, const void *inp, int64_t BT, int64_t C, int64_t R,
+                       int accumulate, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = check_dims(BT, C, R);
+    if (rc != NB_OK) return rc;
+    if (R > 64) return fail(NB_ERR_UNSUPPORTED, "stacked rank must be at most 64");
+    if (!da_stack || !u_stack || !inp) return fail(NB_ERR_INVALID_ARG, "da_stack, u_stack and inp must not be NULL");
+    if (!aligned16(da_stack) || !aligned16(u_stack) || !aligned16(inp))
+        return fail(NB_ERR_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceState *s;
+    if ((rc = get_state(&s)) != NB_OK) return rc;
+    if (BT == 0) {
+        if (!accumulate) NB_CUDA(cudaMemsetAsync(da_stack, 0, static_cast<size_t>(R * C) * 4, stream));
+        return NB_OK;
+    }
+    return run_wgrad_f32(*s, u_stack, inp, da_stack, nullptr, BT, R, C, accumulate, stream);  // dA (+)= u^T . inp
 }
 
 int nb_cast_f32_to_bf16(void *dst, const void *src, int64_t n, void *stream_)

@@ -310,34 +310,62 @@ class LoraStack:
     per layer, base weights frozen, a rank-r adapter beside each (rank-stabilised scale alpha / sqrt(r)).
     A step is every adapted projection forward, then backward in reverse order: dinp through the frozen
     weight and the adapter, fp32 gradients of A and B accumulated over the micro-steps. Same interface
-    as `LinearStack` as far as the benchmark uses it."""
+    as `LinearStack` as far as the benchmark uses it.
+
+    Projections that read the same activations (q, k, v; gate, up) form a group with one input per
+    micro-step. With `stacked=True` (the default) a group's A matrices are rows of one `a_stack`, its
+    down-projections are one rank-R product, and its A gradients one weight-gradient product, so the
+    input is read once per group in each direction; the per-projection `lora_a` / `dlora_a` are row
+    views of the stacks. With `stacked=False` every projection issues the unstacked calls (same tensors,
+    same results)."""
+
+    GROUPS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
 
     def __init__(self, BT: int, micro_steps: int = 1, device="cuda", r: int = 16, alpha: float = 32.0,
                  layers: int = shapes.QWEN3_LAYERS, config_id: int = 6, seed_offset: int = 0,
-                 generate: bool = True):
+                 generate: bool = True, stacked: bool = True):
         self.BT, self.micro_steps, self.device, self.r = BT, micro_steps, device, r
         self.scale = alpha / (r ** 0.5)
         self.wgrad, self.wgrad_stream = False, False
+        self.stacked = stacked
         self.config_id, self.seed_offset = config_id, seed_offset
         self.layers: list[_Layer] = []
+        self.groups: list[list[_Layer]] = []
         idx = 0
         bf, f32 = torch.bfloat16, torch.float32
         for _ in range(layers):
-            for s in shapes.qwen3_lora_projections():
-                L = _Layer(s, idx)
-                L.weight = torch.empty((s.OC, s.C), dtype=bf, device=device)
-                L.lora_a = torch.empty((r, s.C), dtype=bf, device=device)
-                L.lora_b = torch.empty((s.OC, r), dtype=bf, device=device)
-                L.t = torch.empty((BT, r), dtype=bf, device=device)
-                L.u = torch.empty((BT, r), dtype=bf, device=device)
-                L.dlora_a = torch.empty((r, s.C), dtype=f32, device=device)
-                L.dlora_b = torch.empty((s.OC, r), dtype=f32, device=device)
-                L.out = torch.empty((BT, s.OC), dtype=bf, device=device)
-                L.dinp = torch.empty((BT, s.C), dtype=bf, device=device)
-                L.inp = [torch.empty((BT, s.C), dtype=bf, device=device) for _ in range(micro_steps)]
-                L.dout = [torch.empty((BT, s.OC), dtype=bf, device=device) for _ in range(micro_steps)]
-                self.layers.append(L)
-                idx += 1
+            specs = {s.name: s for s in shapes.qwen3_lora_projections()}
+            for names in self.GROUPS:
+                members = []
+                R = r * len(names)
+                C = specs[names[0]].C
+                a_stack = torch.empty((R, C), dtype=bf, device=device)
+                da_stack = torch.empty((R, C), dtype=f32, device=device)
+                t_stack = torch.empty((BT, R), dtype=bf, device=device)
+                u_stack = torch.empty((BT, R), dtype=bf, device=device)
+                inp = [torch.empty((BT, C), dtype=bf, device=device) for _ in range(micro_steps)]
+                for j, name in enumerate(names):
+                    s = specs[name]
+                    assert s.C == C
+                    L = _Layer(s, idx)
+                    L.group_off, L.group_R = j * r, R
+                    L.a_stack, L.da_stack, L.t_stack, L.u_stack = a_stack, da_stack, t_stack, u_stack
+                    L.weight = torch.empty((s.OC, s.C), dtype=bf, device=device)
+                    L.lora_a = a_stack[j * r:(j + 1) * r]          # contiguous rows of the stack
+                    L.dlora_a = da_stack[j * r:(j + 1) * r]
+                    L.lora_b = torch.empty((s.OC, r), dtype=bf, device=device)
+                    L.dlora_b = torch.empty((s.OC, r), dtype=f32, device=device)
+                    # the unstacked calls keep t and u per projection
+                    L.t = torch.empty((BT, r), dtype=bf, device=device)
+                    L.u = torch.empty((BT, r), dtype=bf, device=device)
+                    L.out = torch.empty((BT, s.OC), dtype=bf, device=device)
+                    L.dinp = torch.empty((BT, s.C), dtype=bf, device=device)
+                    L.inp = inp                                     # shared by the group
+                    L.dout = [torch.empty((BT, s.OC), dtype=bf, device=device) for _ in range(micro_steps)]
+                    members.append(L)
+                    self.layers.append(L)
+                    idx += 1
+                self.groups.append(members)
         if generate:
             self.generate_inputs()
 
@@ -346,20 +374,22 @@ class LoraStack:
 
     def generate_inputs(self):
         dev = self.device
-        for L in self.layers:
-            s = L.spec
-            L.weight.copy_(synth.normal(self.seed(L, 1), (s.OC, s.C), s.w_std, dev))
-            L.lora_a.copy_(synth.normal(self.seed(L, 4), (self.r, s.C), 0.02, dev))
-            L.lora_b.copy_(synth.normal(self.seed(L, 5), (s.OC, self.r), 0.02, dev))  # a trained adapter
-            for ms in range(self.micro_steps):
-                L.inp[ms].copy_(synth.normal(self.seed(L, 0, ms), (self.BT, s.C), 1.0, dev))
-                L.dout[ms].copy_(synth.normal(self.seed(L, 3, ms), (self.BT, s.OC), 1e-3, dev))
+        for G in self.groups:
+            for ms in range(self.micro_steps):  # one input per group, seeded by its first member
+                G[0].inp[ms].copy_(synth.normal(self.seed(G[0], 0, ms), (self.BT, G[0].spec.C), 1.0, dev))
+            for L in G:
+                s = L.spec
+                L.weight.copy_(synth.normal(self.seed(L, 1), (s.OC, s.C), s.w_std, dev))
+                L.lora_a.copy_(synth.normal(self.seed(L, 4), (self.r, s.C), 0.02, dev))
+                L.lora_b.copy_(synth.normal(self.seed(L, 5), (s.OC, self.r), 0.02, dev))  # a trained adapter
+                for ms in range(self.micro_steps):
+                    L.dout[ms].copy_(synth.normal(self.seed(L, 3, ms), (self.BT, s.OC), 1e-3, dev))
 
     def input_tensors(self, ms: int):
-        return [t for L in self.layers for t in (L.inp[ms], L.dout[ms])]
+        return [G[0].inp[ms] for G in self.groups] + [L.dout[ms] for L in self.layers]
 
     def gradient_tensors(self):
-        return [g for L in self.layers for g in (L.dlora_a, L.dlora_b)]
+        return [G[0].da_stack for G in self.groups] + [L.dlora_b for L in self.layers]
 
     def flops_per_micro_step(self) -> int:
         """Forward and dinp through the frozen weight, and the six rank-r products of a projection."""
@@ -373,25 +403,45 @@ class LoraStack:
         return L.inp[ms]
 
     def forward(self, ms: int, hook=None):
-        for L in self.layers:
-            s = L.spec
-            if hook:
-                hook("fwd", L, True)
-            nb.nb_lora_linear_forward(L.out, L.t, L.inp[ms], L.weight, None, L.lora_a, L.lora_b, self.scale,
-                                      self.BT, s.C, s.OC, self.r)
-            if hook:
-                hook("fwd", L, False)
+        BT, r = self.BT, self.r
+        for G in self.groups:
+            if self.stacked:
+                L0 = G[0]
+                nb.nb_lora_down_stacked(L0.t_stack, L0.inp[ms], L0.a_stack, self.scale, BT, L0.spec.C, L0.group_R)
+            for L in G:
+                s = L.spec
+                if hook:
+                    hook("fwd", L, True)
+                if self.stacked:
+                    nb.nb_lora_linear_forward_stacked(L.out, L.inp[ms], L.weight, None, L.t_stack, L.lora_b, BT,
+                                                      s.C, s.OC, r, L.group_R, L.group_off)
+                else:
+                    nb.nb_lora_linear_forward(L.out, L.t, L.inp[ms], L.weight, None, L.lora_a, L.lora_b,
+                                              self.scale, BT, s.C, s.OC, r)
+                if hook:
+                    hook("fwd", L, False)
 
     def backward(self, ms: int, hook=None):
+        BT, r = self.BT, self.r
         acc = 1 if ms > 0 else 0
-        for L in reversed(self.layers):
-            s = L.spec
-            if hook:
-                hook("bwd", L, True)
-            nb.nb_lora_linear_backward(L.dinp, L.dlora_a, L.dlora_b, L.u, L.dout[ms], L.inp[ms], L.weight,
-                                       L.lora_a, L.lora_b, L.t, self.scale, self.BT, s.C, s.OC, self.r, acc)
-            if hook:
-                hook("bwd", L, False)
+        for G in reversed(self.groups):
+            for L in reversed(G):
+                s = L.spec
+                if hook:
+                    hook("bwd", L, True)
+                if self.stacked:
+                    nb.nb_lora_linear_backward_stacked(L.dinp, L.dlora_b, L.u_stack, L.dout[ms], L.weight,
+                                                       L.lora_a, L.lora_b, L.t_stack, self.scale, BT, s.C, s.OC,
+                                                       r, L.group_R, L.group_off, acc)
+                else:
+                    nb.nb_lora_linear_backward(L.dinp, L.dlora_a, L.dlora_b, L.u, L.dout[ms], L.inp[ms],
+                                               L.weight, L.lora_a, L.lora_b, L.t, self.scale, BT, s.C, s.OC,
+                                               r, acc)
+                if hook:
+                    hook("bwd", L, False)
+            if self.stacked:
+                L0 = G[0]
+                nb.nb_lora_da_stacked(L0.da_stack, L0.u_stack, L0.inp[ms], BT, L0.spec.C, L0.group_R, acc)
 
     def join(self):
         pass

@@ -168,12 +168,86 @@ def test_adapter_workload_full_batch_sampled(C, OC):
     check_f32(dB, dB_ref, "dlora_b")
 
 
-def test_adapter_stack_driver_two_micro_steps():
+@pytest.mark.parametrize("bias", [False, True])
+@pytest.mark.parametrize("BT,C,ocs,r", [
+    (200, 72, (136, 64, 200), 16),     # three adapters on one input, ragged, one tile
+    (520, 328, (520, 264), 24),        # two adapters, rank 24 (R = 48), several tiles, a CTA pair
+    (300, 1024, (1024, 2048, 8), 8),   # R = 24, many k-blocks before the extension, a tiny projection
+])
+def test_stacked_adapters_equal_the_oracle_per_adapter(BT, C, ocs, r, bias):
+    """Adapters that share an input, stacked: the group's down-projection and A gradient are single
+    products over all adapters, each projection reads and writes its own column slice of t_stack /
+    u_stack. Every result is compared with the oracle of that adapter alone (t and u slices, out,
+    dinp, dB, the rows of dA), with canaries around every buffer, over two accumulating micro-steps."""
+    n = len(ocs)
+    R = n * r
+    scale = 32.0 / math.sqrt(r)
+    inp = gen(1200, (BT, C), 1.0)
+    a_stack = gen(1201, (R, C), 0.02)
+    t_stack = Guarded((BT, R), torch.bfloat16)
+    u_stack = Guarded((BT, R), torch.bfloat16)
+    da_stack = Guarded((R, C), torch.float32, fill=777.0)
+    ws = [gen(1210 + j, (oc, C), 0.02) for j, oc in enumerate(ocs)]
+    bs = [gen(1220 + j, (oc,), 0.02) if bias else None for j, oc in enumerate(ocs)]
+    lbs = [gen(1230 + j, (oc, r), 0.02) for j, oc in enumerate(ocs)]
+    nb.nb_lora_down_stacked(t_stack.t, inp, a_stack, scale, BT, C, R)
+    t_ref, _ = oracle.linear_forward(f32(inp), f32(a_stack))
+    check_bf16(t_stack.t, scale * t_ref, "t_stack")
+    t_stack.check("t_stack")
+    outs, dinps, dBs, dAref, dBref = [], [], [], [None] * n, [None] * n
+    for j, oc in enumerate(ocs):
+        a_j = a_stack[j * r:(j + 1) * r]
+        out = Guarded((BT, oc), torch.bfloat16)
+        nb.nb_lora_linear_forward_stacked(out.t, inp, ws[j], bs[j], t_stack.t, lbs[j], BT, C, oc, r, R, j * r)
+        o_ref = oracle.lora_forward(f32(inp), f32(ws[j]), f32(bs[j]) if bias else None, f32(a_j), f32(lbs[j]), scale)
+        check_bf16(out.t, o_ref, f"out {j}", extra=_rounding_slack(scale * t_ref[:, j * r:(j + 1) * r], f32(lbs[j]).T))
+        out.check(f"out {j}")
+        dinps.append(Guarded((BT, C), torch.bfloat16))
+        dBs.append(Guarded((oc, r), torch.float32, fill=-55.0))
+    for ms in range(2):
+        douts = [gen(1240 + 10 * ms + j, (BT, oc), 1e-3) for j, oc in enumerate(ocs)]
+        u_stack.t.fill_(99.0)  # every column must be rewritten by its own adapter's call
+        for j in reversed(range(n)):
+            oc = ocs[j]
+            a_j = a_stack[j * r:(j + 1) * r]
+            nb.nb_lora_linear_backward_stacked(dinps[j].t, dBs[j].t, u_stack.t, douts[j], ws[j], a_j, lbs[j],
+                                               t_stack.t, scale, BT, C, oc, r, R, j * r, ms)
+            di_ref, dAref[j], dBref[j] = oracle.lora_backward(
+                f32(douts[j]), f32(inp), f32(ws[j]), f32(a_j), f32(lbs[j]), scale,
+                dA=dAref[j], dB=dBref[j], accumulate=ms > 0)
+            u_ref = oracle.linear_backward(f32(douts[j]), None, f32(lbs[j]), want=("dinp",))["dinp"]
+            check_bf16(u_stack.t[:, j * r:(j + 1) * r], scale * u_ref, f"u slice {j}")
+            check_bf16(dinps[j].t, di_ref, f"dinp {j}", extra=_rounding_slack(scale * u_ref, f32(a_j)))
+            check_f32(dBs[j].t, dBref[j], f"dlora_b {j} step {ms}")
+            dinps[j].check(f"dinp {j}")
+            dBs[j].check(f"dlora_b {j}")
+        u_stack.check("u_stack")
+        nb.nb_lora_da_stacked(da_stack.t, u_stack.t, inp, BT, C, R, ms)
+        for j in range(n):
+            check_f32(da_stack.t[j * r:(j + 1) * r], dAref[j], f"dlora_a {j} step {ms}")
+        da_stack.check("da_stack")
+    t_stack.check("t_stack after backward")
+
+
+def test_stacked_rejects_bad_slices():
+    x = torch.zeros((64, 64), dtype=torch.bfloat16, device=DEV)
+    t = torch.zeros((64, 48), dtype=torch.bfloat16, device=DEV)
+    b = torch.zeros((64, 16), dtype=torch.bfloat16, device=DEV)
+    for r, R, off, code in ((16, 48, 40, nb.NB_ERR_INVALID_ARG), (16, 48, 4, nb.NB_ERR_INVALID_ARG),
+                            (16, 72, 0, nb.NB_ERR_UNSUPPORTED), (12, 48, 0, nb.NB_ERR_UNSUPPORTED)):
+        with pytest.raises(nb.NbError) as e:
+            nb.nb_lora_linear_forward_stacked(x, x, x, None, t, b, 64, 64, 64, r, R, off)
+        assert e.value.code == code
+
+
+@pytest.mark.parametrize("stacked", [True, False])
+def test_adapter_stack_driver_two_micro_steps(stacked):
     """The adapter-stage driver: one Qwen3 layer's seven adapted projections, two micro-steps; outputs
-    and dinp of the last micro-step and the accumulated adapter gradients against the oracle."""
+    and dinp of the last micro-step and the accumulated adapter gradients against the oracle, with the
+    adapters of a group stacked (the default) and with one set of calls per projection."""
     from paper_2609_28568_b200.stack import LoraStack
     BT = 384
-    st = LoraStack(BT, micro_steps=2, device=DEV, layers=1)
+    st = LoraStack(BT, micro_steps=2, device=DEV, layers=1, stacked=stacked)
     st.step()
     torch.cuda.synchronize()
     assert [L.spec.name for L in st.layers] == ["q", "k", "v", "o", "gate", "up", "down"]

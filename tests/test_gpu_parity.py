@@ -74,6 +74,37 @@ def test_small_shapes_every_element(BT, C, OC, act):
     run_layer_full(BT, C, OC, act, w_std=0.05, dout_std=1e-3, seed=7 * BT + OC + act)
 
 
+@pytest.mark.parametrize("BT,C,OC", [
+    (129, 8, 8),          # one row past a single tile: the smallest pair problem, one k-block each way
+    (256, 2056, 24),      # one dinp row tile, nine column tiles, a single ragged dweight tile
+    (4100, 72, 136),      # 65 k-blocks of K = BT for dweight, five rows past a tile
+    (1000, 520, 2304),    # more dweight tiles than dinp tiles
+])
+def test_one_launch_backward_edge_shapes(BT, C, OC):
+    """Shapes that stress the work list of the one-launch layer backward (BT > 128: dinp tiles and
+    dweight k-chunks in one kernel): with and without the bias gradient, overwrite then accumulate,
+    and with the producer's GELU derivative in the dinp epilogue; every element against the oracle."""
+    inp, w = gen(300 + BT, (BT, C), 1.0), gen(301 + BT, (OC, C), 0.05)
+    dout, ipre = gen(302 + BT, (BT, OC), 1e-3), gen(303 + BT, (BT, C), 1.0)
+    for bias in (True, False):
+        for fused in (False, True):
+            dinp = Guarded((BT, C), torch.bfloat16)
+            dw = Guarded((OC, C), torch.float32, fill=9.0)
+            db = Guarded((OC,), torch.float32, fill=9.0) if bias else None
+            for acc in (0, 1):
+                nb.nb_linear_backward_ex(dinp.t, dw.t, db.t if db else None, dout, inp, w, None,
+                                         ipre if fused else None, BT, C, OC, nb.ACT_NONE, acc)
+            r = oracle.linear_backward(f32(dout), f32(inp), f32(w), inp_pre=f32(ipre) if fused else None)
+            tag = f"bias={bias} fused={fused}"
+            check_bf16(dinp.t, r["dinp"], "dinp " + tag)
+            check_f32(dw.t, 2.0 * r["dweight"], "dweight " + tag)
+            if db:
+                check_f32(db.t, 2.0 * r["dbias"], "dbias " + tag)
+                db.check("dbias")
+            dinp.check("dinp")
+            dw.check("dweight")
+
+
 def test_integer_inputs_are_exact():
     """Small integers: products and sums are exact in bf16 x bf16 -> fp32, so GPU == oracle exactly.
     Catches any indexing or layout error that a tolerance could hide."""

@@ -56,6 +56,43 @@ def load_peaks():
 
 
 # ------------------------------------------------------------------------------- clocks
+class EnergyMeter:
+    """The GPU's own energy counter (NVML, read-only) around the timed region: joules per step.
+    On a power-capped part the step time follows this figure, not the cycle count."""
+
+    def __init__(self, gpu_id: str):
+        """gpu_id: "GPU-<uuid>" (CUDA and NVML may number the devices differently) or an index."""
+        self.h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            if gpu_id.startswith("GPU-"):
+                try:
+                    self.h = pynvml.nvmlDeviceGetHandleByUUID(gpu_id)
+                except Exception:
+                    self.h = pynvml.nvmlDeviceGetHandleByUUID(gpu_id.encode())
+            else:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(int(gpu_id))
+        except Exception:
+            self.h = None
+
+    def read(self):
+        if self.h is None:
+            return None
+        try:
+            return (self.nv.nvmlDeviceGetTotalEnergyConsumption(self.h) / 1e3, time.time())  # joules, seconds
+        except Exception:
+            return None
+
+    @staticmethod
+    def report(a, b, steps: int):
+        if a is None or b is None or steps <= 0 or b[1] <= a[1]:
+            return None
+        return {"j_per_step": (b[0] - a[0]) / steps, "avg_w": (b[0] - a[0]) / (b[1] - a[1]),
+                "source": "NVML total energy counter around the timed region"}
+
+
 class ClockSampler:
     """nvidia-smi samples (SM clock, throttle reasons) taken while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -405,13 +442,16 @@ def main():
         run_step()  # one untimed replay
     barrier()
     sampler.start()
+    meter = EnergyMeter(gpu_id)
     launches0 = nb.nb_kernel_launches()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    en0 = meter.read()
     ev0.record()
     for _ in range(args.steps):
         run_step()
     ev1.record()
     barrier()
+    energy = EnergyMeter.report(en0, meter.read(), args.steps)
     launches = (launches_per_step * args.steps if launches_per_step is not None
                 else nb.nb_kernel_launches() - launches0)
     nb.nb_check_status()
@@ -513,7 +553,7 @@ def main():
                        "parallelism": (f"dp{world}: fp32 gradient all-reduce in {len(reducer.b.buckets)} buckets "
                                        f"under the last micro-step's backward" if reducer is not None
                                        else f"replicas x{world}, no collective")},
-            "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "clocks": clocks, "energy": energy, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches),
         }
         print(json.dumps(line), flush=True)

@@ -526,6 +526,12 @@ def main():
         "frac_of_sustained_peak": achieved_tf / peaks["bf16_tflops_sustained"],
         "per_call": breakdown,
     }
+    # clock-normalised view: the share of the tensor cores' per-clock capacity (148 SMs x 8192 bf16 flop
+    # per clock on B200) in use at the SM clock sampled during the run; under the power cap the clock
+    # moves against this figure, so neither alone says how good the kernels are
+    if clocks.get("sm_mhz"):
+        roofline["mma_use_per_clock"] = achieved_tf * 1e12 / (props.multi_processor_count * 8192 * clocks["sm_mhz"] * 1e6)
+        roofline["sm_mhz_under_load"] = clocks["sm_mhz"]
 
     # ---- end to end through the C ABI with host buffers (rank-local; max over ranks)
     e2e = None

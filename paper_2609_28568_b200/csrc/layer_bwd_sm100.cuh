@@ -64,10 +64,10 @@ struct LbUnit {
 
 // The sequence of units of one CTA pair; every role of both CTAs walks the same sequence.
 struct LbIter {
-    int r, iD, iW, stage, x, x_end, pair;
+    int r, iD, iW, part, x, x_end, pair;  // part: 0 whole rounds, 1 last D round, 2 W tail, 3 done
     static __host__ __device__ __forceinline__ int imin(int a, int b) { return a < b ? a : b; }
     __host__ __device__ __forceinline__ LbIter(const LayerBwdParams &p, int pair_)
-        : r(0), iD(0), iW(0), stage(0), x(p.w_tail_begin[pair_]), x_end(p.w_tail_begin[pair_ + 1]),
+        : r(0), iD(0), iW(0), part(0), x(p.w_tail_begin[pair_]), x_end(p.w_tail_begin[pair_ + 1]),
           pair(pair_)
     {
     }
@@ -105,7 +105,7 @@ struct LbIter {
     __host__ __device__ __forceinline__ bool next(const LayerBwdParams &p, LbUnit &u)
     {
         while (true) {
-            if (stage == 0) {
+            if (part == 0) {
                 if (r < p.d_rounds + p.w_rounds) {
                     const bool w = ((p.round_is_w >> r) & 1ull) != 0;
                     ++r;
@@ -119,16 +119,16 @@ struct LbIter {
                     }
                     return true;
                 }
-                stage = 1;
+                part = 1;
             }
-            if (stage == 1) {
-                stage = 2;
+            if (part == 1) {
+                part = 2;
                 if (pair < p.d_tail) {
                     d_tile(p, p.d_rounds * p.num_pairs + pair, u);
                     return true;
                 }
             }
-            if (stage == 2) {
+            if (part == 2) {
                 if (x < x_end) {
                     int j = p.w_rounds * p.num_pairs, ko, ulen;
                     if (x < p.w_tail_full) {
@@ -147,7 +147,7 @@ struct LbIter {
                     if (u.kb0 >= u.kb1) continue;
                     return true;
                 }
-                stage = 3;
+                part = 3;
             }
             return false;
         }

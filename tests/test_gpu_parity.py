@@ -105,6 +105,34 @@ def test_one_launch_backward_edge_shapes(BT, C, OC):
             dw.check("dweight")
 
 
+@pytest.mark.parametrize("BT,C,OC,fused", [(8192, 768, 2304, False), (4096, 3072, 768, True)])
+def test_one_launch_backward_is_stable_over_repeated_launches(BT, C, OC, fused):
+    """Sixty launches of the one-launch layer backward, with copies on another stream perturbing the
+    schedule: dinp has no reduction across units and must come out bit for bit the same; dweight and
+    dbias are summed by reduce-adds in varying order and must agree to rounding. A stage handed back
+    too early or a barrier phase off by one shows up here as a rare mismatch."""
+    inp, w = gen(331, (BT, C), 1.0), gen(332, (OC, C), 0.02)
+    dout, ipre = gen(333, (BT, OC), 1e-3), gen(334, (BT, C), 1.0)
+    side = torch.cuda.Stream()
+    ref = None
+    for it in range(60):
+        dinp = torch.empty((BT, C), dtype=torch.bfloat16, device=DEV)
+        dw = torch.full((OC, C), 7.0, dtype=torch.float32, device=DEV)
+        db = torch.full((OC,), 7.0, dtype=torch.float32, device=DEV)
+        if it % 3 == 1:
+            with torch.cuda.stream(side):
+                torch.empty(1 << 24, device=DEV).fill_(1.0)
+        nb.nb_linear_backward_ex(dinp, dw, db, dout, inp, w, None, ipre if fused else None, BT, C, OC,
+                                 nb.ACT_NONE, 0)
+        if ref is None:
+            ref = (dinp, dw, db)
+        else:
+            assert torch.equal(dinp, ref[0]), f"dinp differs at launch {it}"
+            assert rel_frob(f32(dw[:256]), f32(ref[1][:256])) < 1e-5
+            assert rel_frob(f32(db), f32(ref[2])) < 1e-5
+    torch.cuda.synchronize()
+
+
 def test_integer_inputs_are_exact():
     """Small integers: products and sums are exact in bf16 x bf16 -> fp32, so GPU == oracle exactly.
     Catches any indexing or layout error that a tolerance could hide."""

@@ -1041,6 +1041,10 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
     a.splits = 1;
     a.alpha = scale;
     if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    // dB right after u: both stream dout, and what the first pass brought into L2 serves the second
+    if (dlora_b)  // dB [OC, r] (+)= dout^T . t      (t already carries the scale)
+        if ((rc = run_wgrad_f32(*s, dout, t, dlora_b, nullptr, BT, OC, r, accumulate, stream)) != NB_OK)
+            return rc;
     if (dinp) {  // dinp = dout . W + u . A: r extra rows of K
         memset(&a, 0, sizeof(a));
         a.A = dout; a.a_rows = BT; a.a_cols = OC;
@@ -1053,9 +1057,6 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
         a.k2 = static_cast<int>(r);
         if ((rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream)) != NB_OK) return rc;
     }
-    if (dlora_b)  // dB [OC, r] (+)= dout^T . t      (t already carries the scale)
-        if ((rc = run_wgrad_f32(*s, dout, t, dlora_b, nullptr, BT, OC, r, accumulate, stream)) != NB_OK)
-            return rc;
     if (dlora_a)  // dA [r, C] (+)= u^T . inp        (u already carries the scale)
         if ((rc = run_wgrad_f32(*s, u, inp, dlora_a, nullptr, BT, r, C, accumulate, stream)) != NB_OK)
             return rc;
@@ -1164,6 +1165,11 @@ int nb_lora_linear_backward_stacked(void *dinp, void *dlora_b, void *u_stack, co
     a.splits = 1;
     a.alpha = scale;
     if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    // dB right after u: both stream dout, and what the first pass brought into L2 serves the second
+    if (dlora_b)  // dB [OC, r] (+)= dout^T . t_slice
+        if ((rc = run_wgrad_f32(*s, dout, static_cast<const uint16_t *>(t_stack) + off, dlora_b, nullptr, BT, OC, r,
+                                accumulate, stream, static_cast<uint64_t>(R))) != NB_OK)
+            return rc;
     if (dinp) {  // dinp = dout . W + u_slice . A
         memset(&a, 0, sizeof(a));
         a.A = dout; a.a_rows = BT; a.a_cols = OC;
@@ -1176,10 +1182,6 @@ int nb_lora_linear_backward_stacked(void *dinp, void *dlora_b, void *u_stack, co
         a.k2 = static_cast<int>(r);
         if ((rc = launch_gemm_auto<DgradStore1, DgradStore2>(*s, a, stream)) != NB_OK) return rc;
     }
-    if (dlora_b)  // dB [OC, r] (+)= dout^T . t_slice
-        if ((rc = run_wgrad_f32(*s, dout, static_cast<const uint16_t *>(t_stack) + off, dlora_b, nullptr, BT, OC, r,
-                                accumulate, stream, static_cast<uint64_t>(R))) != NB_OK)
-            return rc;
     return NB_OK;
 }
 

@@ -206,7 +206,8 @@ int nb_ce_backward(void *dlogits, const void *logits, const void *lse, const voi
  *     dlora_a (+)= u^T . inp                                    [r, C]    fp32
  * dinp, dlora_a, dlora_b may be NULL (skipped); accumulate as in nb_linear_backward. t and u are
  * rounded to bf16 once each (they are tensor-core operands); everything else follows the
- * conventions at the top of this file.
+ * conventions at the top of this file. When dlora_b is asked for, u and dlora_b come out of one
+ * kernel that reads dout once (both products are bound by that read).
  */
 int nb_lora_linear_forward(void *out, void *t, const void *inp, const void *weight, const void *bias,
                            const void *lora_a, const void *lora_b, float scale, int64_t BT,

@@ -17,6 +17,7 @@
 #include "elementwise.cuh"
 #include "gemm_sm100.cuh"
 #include "layer_bwd_sm100.cuh"
+#include "lora_udb_sm100.cuh"
 
 namespace {
 
@@ -476,6 +477,56 @@ int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight
     }
     if (narrow) return launch_gemm<WgradF32Narrow>(s, a, stream);
     return launch_gemm_auto<WgradF32_1, WgradF32_2>(s, a, stream);
+}
+
+// u = bf16(scale * dy . B) and dB (+)= dy^T . t of one adapted projection from one pass over dy
+// (lora_udb_sm100.cuh). u and t may be column slices of wider tensors (row strides u_ld, t_ld).
+int launch_lora_udb(DeviceState &s, const void *dy, const void *lora_b, const void *t, uint64_t t_ld, void *dlora_b,
+                    void *u, uint64_t u_ld, float scale, int64_t BT, int64_t OC, int64_t r, int accumulate,
+                    cudaStream_t stream)
+{
+    static bool attr_set[kMaxDevices] = {};
+    int dev = 0;
+    NB_CUDA(cudaGetDevice(&dev));
+    if (!attr_set[dev]) {
+        NB_CUDA(cudaFuncSetAttribute(lora_udb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(kUdbSmemBytes)));
+        attr_set[dev] = true;
+    }
+    CUtensorMap tDy, tB, tT, tDb;
+    int rc;
+    if ((rc = get_tmap(s, &tDy, dy, BT, OC, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tB, lora_b, OC, r, 0, 64)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tT, t, BT, r, 0, 64, t_ld)) != NB_OK) return rc;
+    if ((rc = get_tmap(s, &tDb, dlora_b, OC, r, 1, 32)) != NB_OK) return rc;
+    // every panel reduce-adds its share, so a fresh gradient starts from zero
+    if (!accumulate) NB_CUDA(cudaMemsetAsync(dlora_b, 0, static_cast<size_t>(OC * r) * 4, stream));
+    UdbParams p;
+    memset(&p, 0, sizeof(p));
+    p.BT = static_cast<int>(BT);
+    p.OC = static_cast<int>(OC);
+    p.r = static_cast<int>(r);
+    p.panels = static_cast<int>((BT + 127) / 128);
+    p.tiles = static_cast<int>((OC + 127) / 128);
+    p.want_db = 1;
+    p.alpha = scale;
+    p.u = static_cast<__nv_bfloat16 *>(u);
+    p.u_ld = static_cast<int>(u_ld);
+    p.status = s.status;
+    p.timeout_ns = kDefaultTimeoutNs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(p.panels < s.num_sms ? p.panels : s.num_sms));
+    cfg.blockDim = dim3(kUdbThreads);
+    cfg.dynamicSmemBytes = kUdbSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attrs[1];
+    attrs[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = dependent_launch_allowed(stream) ? 1 : 0;
+    NB_CUDA(cudaLaunchKernelEx(&cfg, lora_udb_kernel, tDy, tB, tT, tDb, p));
+    ++g_launches;
+    return NB_OK;
 }
 
 // ----------------------------------------------------------------------------- one launch per layer backward
@@ -1033,14 +1084,22 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
         return NB_OK;
     }
     GemmArgs a;
-    memset(&a, 0, sizeof(a));  // u = scale * dout . B   (B [OC, r] read as an MN-major operand)
-    a.A = dout; a.a_rows = BT; a.a_cols = OC;
-    a.B = lora_b; a.b_rows = OC; a.b_cols = r;
-    a.D = u; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0;
-    a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
-    a.splits = 1;
-    a.alpha = scale;
-    if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    static const bool fused_udb = env_int("NB_LORA_FUSED", 1) != 0;
+    if (fused_udb && dlora_b) {  // u and dB from one pass over dout
+        if ((rc = launch_lora_udb(*s, dout, lora_b, t, 0, dlora_b, u, static_cast<uint64_t>(r), scale, BT, OC, r,
+                                  accumulate, stream)) != NB_OK)
+            return rc;
+        dlora_b = nullptr;
+    } else {
+        memset(&a, 0, sizeof(a));  // u = scale * dout . B   (B [OC, r] read as an MN-major operand)
+        a.A = dout; a.a_rows = BT; a.a_cols = OC;
+        a.B = lora_b; a.b_rows = OC; a.b_cols = r;
+        a.D = u; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0;
+        a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
+        a.splits = 1;
+        a.alpha = scale;
+        if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    }
     // dB right after u: both stream dout, and what the first pass brought into L2 serves the second
     if (dlora_b)  // dB [OC, r] (+)= dout^T . t      (t already carries the scale)
         if ((rc = run_wgrad_f32(*s, dout, t, dlora_b, nullptr, BT, OC, r, accumulate, stream)) != NB_OK)
@@ -1157,14 +1216,23 @@ int nb_lora_linear_backward_stacked(void *dinp, void *dlora_b, void *u_stack, co
     }
     uint16_t *u_slice = static_cast<uint16_t *>(u_stack) + off;
     GemmArgs a;
-    memset(&a, 0, sizeof(a));  // u_slice = scale * dout . B
-    a.A = dout; a.a_rows = BT; a.a_cols = OC;
-    a.B = lora_b; a.b_rows = OC; a.b_cols = r;
-    a.D = u_slice; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0; a.d_ld = R;
-    a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
-    a.splits = 1;
-    a.alpha = scale;
-    if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    static const bool fused_udb = env_int("NB_LORA_FUSED", 1) != 0;
+    if (fused_udb && dlora_b) {  // u_slice and dB from one pass over dout
+        if ((rc = launch_lora_udb(*s, dout, lora_b, static_cast<const uint16_t *>(t_stack) + off, static_cast<uint64_t>(R),
+                                  dlora_b, u_slice, static_cast<uint64_t>(R), scale, BT, OC, r, accumulate,
+                                  stream)) != NB_OK)
+            return rc;
+        dlora_b = nullptr;
+    } else {
+        memset(&a, 0, sizeof(a));  // u_slice = scale * dout . B
+        a.A = dout; a.a_rows = BT; a.a_cols = OC;
+        a.B = lora_b; a.b_rows = OC; a.b_cols = r;
+        a.D = u_slice; a.d_rows = BT; a.d_cols = r; a.d_dtype = 0; a.d_ld = R;
+        a.M = static_cast<int>(BT); a.N = static_cast<int>(r); a.K = static_cast<int>(OC);
+        a.splits = 1;
+        a.alpha = scale;
+        if ((rc = launch_gemm<DgradStoreNarrow>(*s, a, stream)) != NB_OK) return rc;
+    }
     // dB right after u: both stream dout, and what the first pass brought into L2 serves the second
     if (dlora_b)  // dB [OC, r] (+)= dout^T . t_slice
         if ((rc = run_wgrad_f32(*s, dout, static_cast<const uint16_t *>(t_stack) + off, dlora_b, nullptr, BT, OC, r,

@@ -10,7 +10,7 @@
 //     columns: the panel's u, accumulated in TMEM over all tiles of the panel;
 //   - as an MN-major A operand (M = the 128 columns, K = the 128 rows) against the panel's rows of
 //     t: this panel's whole contribution to 128 rows of dB, which the epilogue reduce-adds into
-//     dB at once (two TMEM buffers, so the next tile's MMAs do not wait for it).
+//     dB at once (four TMEM buffers, so the next tiles' MMAs do not wait for it).
 // A tile is fetched as four 64 x 64 boxes with 128-byte rows and the 128-byte swizzle; "row r,
 // 64 columns" is at the same place whether the tensor core walks the tile by rows or by columns,
 // which is what lets one copy serve both products.
@@ -32,7 +32,8 @@ constexpr uint32_t kUdbOffT = kUdbOffB + kUdbStages * kUdbBBytes;
 constexpr uint32_t kUdbOffStg = kUdbOffT + kUdbBBytes;          // 4 warps x 2 boxes of 4 KB
 constexpr uint32_t kUdbOffBar = kUdbOffStg + 4 * 2 * 4096;
 constexpr uint32_t kUdbSmemBytes = kUdbOffBar + 256;
-constexpr uint32_t kUdbTmemCols = 256;  // u: 64 columns; two dB buffers of 64
+constexpr int kUdbDbBufs = 4;
+constexpr uint32_t kUdbTmemCols = 512;  // u: 64 columns; four dB buffers of 64
 
 struct UdbParams {
     int BT, OC, r;
@@ -61,17 +62,18 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
     if (!smem_ok && threadIdx.x == 0 && atomicCAS(p.status, 0, kStatusBadSmem) == 0)
         p.status[2] = static_cast<int>(blockIdx.x);
 
-    // barriers: full[S], empty[S], t_full, t_empty, u_full, u_empty, db_full[2], db_empty[2]
+    // barriers: full[S], empty[S], t_full, t_empty, u_full, u_empty, db_full[NB], db_empty[NB]
     constexpr int S = kUdbStages;
+    constexpr int NB = kUdbDbBufs;
     const uint32_t bar0 = smem + kUdbOffBar;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (S + s); };
     const uint32_t t_full = bar0 + 8u * (2 * S), t_empty = bar0 + 8u * (2 * S + 1);
     const uint32_t u_full = bar0 + 8u * (2 * S + 2), u_empty = bar0 + 8u * (2 * S + 3);
     auto dbfull_bar = [&](int b) { return bar0 + 8u * (2 * S + 4 + b); };
-    auto dbempty_bar = [&](int b) { return bar0 + 8u * (2 * S + 6 + b); };
+    auto dbempty_bar = [&](int b) { return bar0 + 8u * (2 * S + 4 + NB + b); };
     const uint32_t tmem_slot = bar0 + 240, abort_addr = bar0 + 244;
-    static_assert(8 * (2 * S + 8) <= 240, "barrier region");
+    static_assert(8 * (2 * S + 4 + 2 * NB) <= 240, "barrier region");
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -82,7 +84,7 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
         ptx::mbar_init(t_empty, 1);   // the issuer's commit after a panel's last tile
         ptx::mbar_init(u_full, 1);
         ptx::mbar_init(u_empty, 4);   // one arrive per epilogue warp
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < NB; ++b) {
             ptx::mbar_init(dbfull_bar(b), 1);
             ptx::mbar_init(dbempty_bar(b), 4);
         }
@@ -199,7 +201,7 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                     ptx::umma_commit<1>(empty_bar(stage));
                     if (p.want_db) {
                         ptx::umma_commit<1>(dbfull_bar(buf));
-                        if (++buf == 2) {
+                        if (++buf == NB) {
                             buf = 0;
                             bphase ^= 1u;
                         }
@@ -239,7 +241,16 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                     // rows = 32 of the tile's 128 columns of dy (rows of dB), columns = r (<= 64)
                     for (int c = 0; c < p.r; c += 32) {
                         uint32_t r32[32];
-                        ptx::tmem_ld_32x32_wait(t_acc + static_cast<uint32_t>(c), r32);
+                        if (p.r <= 16) {  // half the columns are enough; the rest of the box is clipped by the copy
+                            uint32_t r16[16];
+                            ptx::tmem_ld_32x16_wait(t_acc, r16);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) r32[i] = r16[i];
+#pragma unroll
+                            for (int i = 16; i < 32; ++i) r32[i] = 0u;
+                        } else {
+                            ptx::tmem_ld_32x32_wait(t_acc + static_cast<uint32_t>(c), r32);
+                        }
                         const uint32_t fb = stg + (box & 1u) * 4096u;
                         ++box;
                         ptx::bulk_wait_group_read<1>();
@@ -260,7 +271,7 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(dbempty_bar(buf));
                     __syncwarp();
-                    if (++buf == 2) {
+                    if (++buf == NB) {
                         buf = 0;
                         bphase ^= 1u;
                     }

@@ -59,7 +59,7 @@ int nbo_reduce_dbias_f64(double *dbias, const float *dout, int64_t BT, int64_t O
 
 /*
  * fp32 -> bf16, round to nearest, ties to even (the master-weight cast done once per optimizer
- * step; paper: Results/Speed, the table of levers, "master-cast reuse across micro-steps").
+ * step; paper: Results/Speed, the table of levers, the row on reusing the cast across micro-steps).
  * Written on the bit patterns: keep the top 16 bits, add one when the discarded half is above
  * one half of the last kept bit, or exactly one half and the kept value is odd. Infinities stay,
  * a carry out of the largest finite value gives infinity, NaN stays NaN (quiet, sign kept).
@@ -82,8 +82,8 @@ void nbo_cast_f32_bf16(uint16_t *dst, const float *src, int64_t n)
 }
 
 /*
- * Cross-entropy of the head's logits over the first V of Vp columns (paper: Figure 1, "cross-entropy
- * over the first 50,257; padding rows get no probability and no gradient"; loss in f32).
+ * Cross-entropy of the head's logits over the first V of Vp columns (paper: Figure 1, the loss box:
+ * only the 50,257 real tokens take part, the padding columns get neither probability nor gradient; loss in f32).
  *   lse[i]       = log sum_{j<V} exp(logits[i,j])
  *   loss[i]      = lse[i] - logits[i, target[i]]
  *   dlogits[i,j] = gscale * (exp(logits[i,j] - lse[i]) - [j == target[i]])   for j <  V

@@ -10,6 +10,7 @@ import os
 import socket
 import subprocess
 import sys
+import time
 
 
 def free_port() -> int:
@@ -43,12 +44,13 @@ def spawn_ranks(n: int, argv: list[str], python: str | None = None, env_extra: d
         procs.append(subprocess.Popen([python or sys.executable, *argv], env=env,
                                       stdout=None if r == 0 else sys.stderr))
     rc = 0
+    deadline = None if timeout is None else time.monotonic() + timeout
     try:
         pending = list(procs)
         while pending:
             for p in list(pending):
                 try:
-                    code = p.wait(timeout=0.2 if timeout is None else min(0.2, timeout))
+                    code = p.wait(timeout=0.2)
                 except subprocess.TimeoutExpired:
                     continue
                 pending.remove(p)
@@ -56,13 +58,11 @@ def spawn_ranks(n: int, argv: list[str], python: str | None = None, env_extra: d
                     rc = max(rc, code if code > 0 else 1)
                     for q in pending:   # one rank failed: the others would wait at a barrier for ever
                         q.terminate()
-            if timeout is not None:
-                timeout -= 0.2
-                if timeout <= 0 and pending:
-                    for q in pending:
-                        q.terminate()
-                    rc = max(rc, 124)
-                    timeout = None
+            if deadline is not None and pending and time.monotonic() > deadline:
+                for q in pending:
+                    q.terminate()
+                rc = max(rc, 124)
+                deadline = None
     finally:
         for p in procs:
             if p.poll() is None:

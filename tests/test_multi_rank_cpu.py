@@ -67,7 +67,7 @@ assert os.environ["MASTER_ADDR"] == "127.0.0.1" and int(os.environ["LOCAL_RANK"]
 dist.init_process_group("gloo", rank=rank, world_size=world)
 t = torch.tensor([10.0 * (rank + 1)], dtype=torch.float64)
 dist.all_reduce(t, op=dist.ReduceOp.MAX)
-os.write(1, b"noise from rank %d\n" % rank) if rank else None  # one write: lines of two ranks cannot interleave
+os.write(1, b"noise from rank %d\\n" % rank) if rank else None  # one write: lines of two ranks cannot interleave
 if rank == 0:
     print(json.dumps({"n_gpus": world, "slowest": float(t.item()), "argv": sys.argv[1:]}))
 dist.destroy_process_group()

@@ -13,7 +13,9 @@
 //     dB at once (four TMEM buffers, so the next tiles' MMAs do not wait for it).
 // A tile is fetched as four 64 x 64 boxes with 128-byte rows and the 128-byte swizzle; "row r,
 // 64 columns" is at the same place whether the tensor core walks the tile by rows or by columns,
-// which is what lets one copy serve both products.
+// which is what lets one copy serve both products. The panels walk the column tiles in rotated
+// orders (panel pn starts at tile pn mod tiles), so that at any moment the CTAs work on different
+// rows of B and dB.
 //
 // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue (TMEM lane quarter = warp % 4).
 // Every wait is bounded as in gemm_kernel; on expiry the kernel records it and leaves.
@@ -132,7 +134,10 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                     ptx::mbar_expect_tx(full_bar(stage), kUdbABytes + kUdbBBytes);
                     const uint32_t sa = smem + kUdbOffA + stage * kUdbABytes;
                     const uint32_t sb = smem + kUdbOffB + stage * kUdbBBytes;
-                    const int c0 = j * 128;
+                    // Panel pn starts at column tile pn % tiles and wraps around: with every CTA on
+                    // tile 0 at the same time, all of them fetched the same rows of B and reduce-added
+                    // into the same rows of dB at once (a quarter of the kernel's time went there).
+                    const int c0 = ((j + pn) % p.tiles) * 128;
                     // dy tile: columns c0..+63 for rows 0..127 (16 KB), then columns c0+64..+127
                     ptx::tma_load_2d(sa, &tmDy, full_bar(stage), c0, m0);
                     ptx::tma_load_2d(sa + 8192u, &tmDy, full_bar(stage), c0, m0 + 64);
@@ -261,7 +266,7 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (ptx::elect_one()) {
-                            const int y = j * 128 + q * 32;
+                            const int y = ((j + pn) % p.tiles) * 128 + q * 32;  // the producer's tile order
                             if (y < p.OC) ptx::tma_reduce_add_2d(&tmDb, fb, c, y);
                             ptx::bulk_commit_group();
                         }

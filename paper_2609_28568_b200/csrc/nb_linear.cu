@@ -422,7 +422,9 @@ int launch_dbias(DeviceState &s, float *dbias, const void *dz, int64_t BT, int64
     if (!accumulate) NB_CUDA(cudaMemsetAsync(dbias, 0, static_cast<size_t>(OC) * 4, stream));
     if (BT == 0) return NB_OK;
     const int col_blocks = static_cast<int>((OC + kDbiasCols - 1) / kDbiasCols);
-    long long want_row_blocks = (6ll * s.num_sms + col_blocks - 1) / col_blocks;
+    // about three blocks per SM: with six (or one) the same kernel was 15-25 % slower on the stack's
+    // shapes (measured: 16.6 us against 19.2 us for 16384 x 2304)
+    long long want_row_blocks = (3ll * s.num_sms + col_blocks - 1) / col_blocks;
     long long rows_per_block = (BT + want_row_blocks - 1) / want_row_blocks;
     rows_per_block = ((rows_per_block + 127) / 128) * 128;  // a block sweeps 128 rows per iteration
     if (rows_per_block < 128) rows_per_block = 128;

@@ -312,7 +312,7 @@ def main():
     ap.add_argument("--workload", default="gpt2_124m_stack", choices=sorted(WORKLOADS))
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from the host in the timed region instead of replaying a CUDA graph")
     ap.add_argument("--two-streams", action="store_true",
@@ -570,7 +570,7 @@ def main():
         dist.destroy_process_group()
 
 
-def measure_e2e(torch, nb, stack, args, dist, dev, flops_step, world):
+def measure_e2e(torch, nb, stack, args, dist, dev, flops_step, world, return_host=False):
     """The same step with every micro-step's inputs copied from pinned host memory inside the timed
     region, and the accumulated gradients read back to the host at the end of each step."""
     host_in = []
@@ -587,26 +587,42 @@ def measure_e2e(torch, nb, stack, args, dist, dev, flops_step, world):
     host_out = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True) for g in grads]
     d2h = sum(g.numel() * g.element_size() for g in grads)
     copy_stream = torch.cuda.Stream(device=dev)
+    d2h_stream = torch.cuda.Stream(device=dev)
     main = torch.cuda.current_stream()
+    n_ms = stack.micro_steps
+    used = [None] * n_ms   # event: the previous step's micro-step ms has finished with its input buffers
+    read = [None]          # event: the previous step's gradients have been read back
 
     def one_step():
-        # inputs of micro-step i+1 are copied while micro-step i computes
+        # Three queues: inputs of micro-step ms go to the device as soon as the previous step's micro-step
+        # ms has released those buffers (so the copies of step i+1 run under the compute of step i),
+        # the micro-steps wait for their own inputs, and the gradients of a step are read back on a
+        # third stream while the next step's inputs already arrive (PCIe carries both directions).
         ready = []
-        for ms in range(stack.micro_steps):
+        for ms in range(n_ms):
             with torch.cuda.stream(copy_stream):
+                if used[ms] is not None:
+                    copy_stream.wait_event(used[ms])
                 for h, t in zip(host_in[ms], stack.input_tensors(ms)):
                     t.copy_(h, non_blocking=True)
                 e = torch.cuda.Event()
                 e.record(copy_stream)
                 ready.append(e)
-        for ms in range(stack.micro_steps):
+        for ms in range(n_ms):
             main.wait_event(ready[ms])
+            if ms == 0 and read[0] is not None:
+                main.wait_event(read[0])   # micro-step 0 overwrites the gradients
             stack.micro_step(ms)
-        for g, h in zip(grads, host_out):
-            h.copy_(g, non_blocking=True)
+            used[ms] = torch.cuda.Event()
+            used[ms].record(main)
+        with torch.cuda.stream(d2h_stream):
+            d2h_stream.wait_event(used[n_ms - 1])
+            for g, h in zip(grads, host_out):
+                h.copy_(g, non_blocking=True)
+            read[0] = torch.cuda.Event()
+            read[0].record(d2h_stream)
 
     torch.cuda.synchronize()
-    copy_stream.wait_stream(main)
     one_step()  # warm-up
     torch.cuda.synchronize()
     if dist is not None:
@@ -615,18 +631,21 @@ def measure_e2e(torch, nb, stack, args, dist, dev, flops_step, world):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.e2e_steps):
-        copy_stream.wait_stream(main)  # the next step's copies may not overwrite inputs still in use
         one_step()
+    main.wait_stream(d2h_stream)  # the last step's gradients are on the host before the clock stops
+    main.wait_stream(copy_stream)
     ev1.record()
     torch.cuda.synchronize()
     wall_ms = (time.perf_counter() - t0) * 1e3
     ms = max_over_ranks(max(ev0.elapsed_time(ev1), wall_ms) / args.e2e_steps, dist, dev)
     nb.nb_check_status()
-    return {"value": world * flops_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+    result = {"value": world * flops_step / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ms,
             "steps": args.e2e_steps,
-            "note": "inputs of each micro-step copied from pinned host memory on a copy stream, "
-                    "gradients read back to pinned host memory, all inside the timed region"}
+            "note": "inputs of each micro-step copied from pinned host memory on a copy stream (the next "
+                    "step's copies start as soon as the buffers are free), gradients read back to pinned "
+                    "host memory on a third stream, all inside the timed region"}
+    return (result, host_out) if return_host else result
 
 
 if __name__ == "__main__":

@@ -925,3 +925,28 @@ def test_timed_path_full_stack_graph_replay_sampled_against_the_oracle():
             if L.dbias is not None:
                 ref_b = sum(oracle.reduce_dbias(f32(L.dout[ms])) for ms in range(MS))
                 check_f32(L.dbias, ref_b, "stack " + s.name + " dbias over micro-steps")
+
+
+def test_end_to_end_path_of_the_bench_returns_the_step_gradients():
+    """The bench's end-to-end leg streams every micro-step's inputs from pinned host memory on a copy
+    stream, computes on the main stream and reads the gradients back on a third one, steps overlapping.
+    What arrives on the host after three such steps must be the gradients of one plain step (the inputs
+    are the same every step; fp32 sums may differ in their last bits)."""
+    import argparse
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    from paper_2609_28568_b200.stack import LinearStack
+    stack = LinearStack("gpt2_block", 1024, 3, device=torch.device("cuda", 0), config_id=2)
+    stack.step()
+    torch.cuda.synchronize()
+    want = [g.clone() for g in stack.gradient_tensors()]
+    for g in stack.gradient_tensors():
+        g.fill_(float("nan"))
+    args = argparse.Namespace(e2e_steps=3)
+    res, host = bench.measure_e2e(torch, nb, stack, args, None, torch.device("cuda", 0), 1.0, 1, return_host=True)
+    assert res["h2d_bytes_per_step"] > 0 and res["d2h_bytes_per_step"] == sum(w.numel() * 4 for w in want)
+    for h, w in zip(host, want):
+        assert torch.isfinite(h).all()
+        assert rel_frob(h.numpy(), f32(w)) < 1e-5

@@ -144,3 +144,41 @@ def test_layer_backward_plan_covers_every_unit_once(L):
                     # level to within a few k-blocks (cuts are rounded to four, a cut unit pays
                     # its allowance twice)
                     assert max(load) - min(load) <= 16, (BT, C, OC, pairs, gelu, max(load), min(load))
+
+
+def test_layer_backward_plan_on_drawn_shapes(L):
+    """The same partition property on 200 drawn problems (seeded): row counts from just past one tile to
+    70,000, widths from 8 to 6144, several pair counts. Either the planner declines (more rounds than its
+    order mask holds) or every dinp tile appears once and every (dweight tile, k-block) exactly once."""
+    import numpy as np
+    rng = np.random.default_rng(20260928)
+    declined = 0
+    for case in range(200):
+        BT = int(rng.integers(129, 70_000)) if case % 4 else int(rng.choice((129, 256, 257, 4096, 16384, 65536)))
+        C = 8 * int(rng.integers(1, 769))
+        OC = 8 * int(rng.integers(1, 769))
+        pairs = int(rng.choice((74, 66, 33, 7)))
+        gelu = bool(rng.integers(0, 2))
+        try:
+            hdr, recs = binding.nb_debug_layer_bwd_plan(BT, C, OC, pairs, gelu)
+        except binding.NbError as e:
+            assert e.code == binding.NB_ERR_UNSUPPORTED
+            declined += 1
+            continue
+        dtm, dtn, dkb, wtm, wtn, wkb, kbc, rounds = hdr
+        tag = (BT, C, OC, pairs, gelu)
+        assert (dtm, dtn, dkb) == (-(-BT // 256), -(-C // 256), -(-OC // 64)), tag
+        assert (wtm, wtn, wkb) == (-(-OC // 256), -(-C // 256), -(-BT // 64)), tag
+        d_seen = np.zeros((dtm, dtn), dtype=np.int64)
+        w_cov = np.zeros((wtm, wtn, wkb), dtype=np.int64)
+        for pr, is_w, m, n, kb0, kb1 in recs:
+            assert 0 <= pr < pairs and kb0 < kb1, tag
+            if is_w:
+                assert kb1 <= wkb, tag
+                w_cov[m, n, kb0:kb1] += 1
+            else:
+                assert (kb0, kb1) == (0, dkb), tag
+                d_seen[m, n] += 1
+        assert (d_seen == 1).all(), tag
+        assert (w_cov == 1).all(), tag
+    assert declined < 100   # the drawn set mostly exercises the planner, not its refusal

@@ -950,3 +950,23 @@ def test_end_to_end_path_of_the_bench_returns_the_step_gradients():
     for h, w in zip(host, want):
         assert torch.isfinite(h).all()
         assert rel_frob(h.numpy(), f32(w)) < 1e-5
+
+
+def test_layer_backward_beyond_the_one_launch_schedule_falls_back_to_separate_launches():
+    """A layer with more dinp tiles than the one-launch schedule's round mask holds (79 x 64 tiles for 74
+    CTA pairs) is declined by the planner; the call must then issue dinp and dweight as launches of their
+    own and still give the oracle's results (sampled rows, columns and a stratified grid; dbias whole)."""
+    BT, C, OC = 20000, 16384, 8
+    with pytest.raises(nb.NbError):
+        nb.nb_debug_layer_bwd_plan(BT, C, OC, 74, False)
+    inp, w = gen(7001, (BT, C), 1.0), gen(7002, (OC, C), 0.05)
+    dout = gen(7003, (BT, OC), 1e-3)
+    dinp = Guarded((BT, C), torch.bfloat16)
+    dw = Guarded((OC, C), torch.float32, fill=4.0)
+    db = Guarded((OC,), torch.float32, fill=4.0)
+    before = nb.nb_kernel_launches()
+    nb.nb_linear_backward_ex(dinp.t, dw.t, db.t, dout, inp, w, None, None, BT, C, OC, nb.ACT_NONE, 0)
+    assert nb.nb_kernel_launches() - before == 2   # dinp, and dweight with the bias gradient inside
+    _bwd_sampled("fallback", dout, inp, w, dinp.t, dw.t, db.t, seed=77)
+    for g, n in ((dinp, "dinp"), (dw, "dweight"), (db, "dbias")):
+        g.check(n)

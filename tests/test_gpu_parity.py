@@ -970,3 +970,46 @@ def test_layer_backward_beyond_the_one_launch_schedule_falls_back_to_separate_la
     _bwd_sampled("fallback", dout, inp, w, dinp.t, dw.t, db.t, seed=77)
     for g, n in ((dinp, "dinp"), (dw, "dweight"), (db, "dbias")):
         g.check(n)
+
+
+def test_release_and_workspace_growth_refused_during_capture():
+    """nb_release drops the library's device state (workspace, status word, tensor-map cache); the next
+    call builds it again. With the workspace back at zero, an own-activation backward issued while its
+    stream is being captured would have to allocate: it is refused with a message naming
+    nb_workspace_reserve, the capture survives and replays what it recorded, and after a reserve the same
+    call captures and gives the oracle's bias gradient."""
+    nb.nb_check_status()
+    nb.nb_release()
+    BT, OC = 1024, 520
+    dout, pre = gen(7101, (BT, OC), 1e-3), gen(7102, (BT, OC), 1.0)
+    x, w = gen(7103, (BT, 64), 1.0), gen(7104, (OC, 64), 0.05)
+    out = torch.zeros((BT, OC), dtype=torch.bfloat16, device=DEV)
+    db = torch.zeros((OC,), dtype=torch.float32, device=DEV)
+    nb.nb_linear_forward_ex(out, None, x, w, None, BT, 64, OC, nb.ACT_NONE)   # state and tensor maps exist again
+    torch.cuda.synchronize()
+    want_out = out.clone()
+    out.zero_()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            nb.nb_linear_forward_ex(out, None, x, w, None, BT, 64, OC, nb.ACT_NONE)
+            with pytest.raises(nb.NbError) as ei:
+                nb.nb_linear_backward_ex(None, None, db, dout, None, None, pre, None, BT, 8, OC, nb.ACT_GELU, 0)
+            assert ei.value.code == nb.NB_ERR_UNSUPPORTED and "nb_workspace_reserve" in str(ei.value)
+    torch.cuda.current_stream().wait_stream(s)
+    g.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, want_out)
+    nb.nb_workspace_reserve(BT * OC * 2)
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        g2 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g2, stream=s):
+            nb.nb_linear_backward_ex(None, None, db, dout, None, None, pre, None, BT, 8, OC, nb.ACT_GELU, 0)
+    torch.cuda.current_stream().wait_stream(s)
+    g2.replay()
+    torch.cuda.synchronize()
+    dz = f32(dout).astype(np.float64) * oracle.gelu_grad(f32(pre).astype(np.float64))
+    check_f32(db, oracle.reduce_dbias(dz.astype(np.float32)), "dbias through a captured own-activation backward")

@@ -320,6 +320,9 @@ def main():
                          "stream, one launch per layer backward; the two arrangements time the same on a "
                          "power-capped part)")
     ap.add_argument("--one-stream", action="store_true", help="accepted for compatibility: this is the default")
+    ap.add_argument("--lora-unfused", action="store_true",
+                    help="qwen3_lora: one set of calls per projection (seven per layer) instead of one per group "
+                         "of projections that share an input (q_k_v, o, gate_up, down)")
     ap.add_argument("--dp", action="store_true",
                     help="data parallel instead of replicas: the same weights on every rank, its own rows, and "
                          "the fp32 gradients all-reduced (NCCL) in buckets under the last micro-step's backward; "
@@ -366,7 +369,8 @@ def main():
         from paper_2609_28568_b200.stack import LoraStack
         if args.dp:
             raise SystemExit("--dp is wired for the dense stacks only")
-        stack = LoraStack(BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank)
+        stack = LoraStack(BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
+                          fused=not args.lora_unfused)
     else:
         stack = LinearStack(model, BT, micro_steps, device=dev, config_id=cfg_id, seed_offset=rank,
                             wgrad=wgrad, shared_weights=args.dp,

@@ -32,7 +32,7 @@ def soak(workload: str = "gpt2", replays: int = 1000, every: int = 100, device: 
     if workload == "gpt2":
         stack = LinearStack("gpt2", 16384, 4, device=dev, config_id=4)
     elif workload == "qwen3_lora":
-        stack = LoraStack(16384, 1, device=dev, config_id=5)
+        stack = LoraStack(16384, 1, device=dev, config_id=6, fused=True)
     else:
         raise ValueError("workload must be gpt2 or qwen3_lora")
     for _ in range(3):

@@ -317,17 +317,28 @@ class LoraStack:
     down-projections are one rank-R product, and its A gradients one weight-gradient product, so the
     input is read once per group in each direction; the per-projection `lora_a` / `dlora_a` are row
     views of the stacks. With `stacked=False` every projection issues the unstacked calls (same tensors,
-    same results)."""
+    same results).
+
+    With `fused=True` the projections of a group are ONE linear layer, the way such layers are usually
+    laid out (a qkv projection, a gate_up projection): the members' weights are the rows of one
+    `weight`, their outputs the columns of one `out`, and their B matrices the diagonal blocks of one
+    `lora_b` [sum of OC, R] whose other blocks are zero, so that `t_stack @ lora_b.T` adds to each
+    member's columns exactly its own adapter term. The same stacked calls then run once per group
+    (rank R): one forward product, one u / dB pass, one dinp product (the sum of the members' input
+    gradients, which is what the layer below needs) and one dA product. `members` of a fused layer
+    lists (spec, row offset, index used for seeding); the off-diagonal blocks of `dlora_b` receive
+    values that belong to no parameter and are ignored."""
 
     GROUPS = (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))
 
     def __init__(self, BT: int, micro_steps: int = 1, device="cuda", r: int = 16, alpha: float = 32.0,
                  layers: int = shapes.QWEN3_LAYERS, config_id: int = 6, seed_offset: int = 0,
-                 generate: bool = True, stacked: bool = True):
+                 generate: bool = True, stacked: bool = True, fused: bool = False):
         self.BT, self.micro_steps, self.device, self.r = BT, micro_steps, device, r
         self.scale = alpha / (r ** 0.5)
         self.wgrad, self.wgrad_stream = False, False
-        self.stacked = stacked
+        self.stacked = stacked or fused
+        self.fused = fused
         self.config_id, self.seed_offset = config_id, seed_offset
         self.layers: list[_Layer] = []
         self.groups: list[list[_Layer]] = []
@@ -344,11 +355,33 @@ class LoraStack:
                 t_stack = torch.empty((BT, R), dtype=bf, device=device)
                 u_stack = torch.empty((BT, R), dtype=bf, device=device)
                 inp = [torch.empty((BT, C), dtype=bf, device=device) for _ in range(micro_steps)]
+                if fused:
+                    OCt = sum(specs[n].OC for n in names)
+                    L = _Layer(shapes.LinearSpec("_".join(names) if len(names) > 1 else names[0], C, OCt, False),
+                               idx)
+                    L.rank, L.group_off, L.group_R = R, 0, R
+                    L.a_stack, L.da_stack, L.t_stack, L.u_stack = a_stack, da_stack, t_stack, u_stack
+                    L.weight = torch.empty((OCt, C), dtype=bf, device=device)
+                    L.lora_a, L.dlora_a = a_stack, da_stack
+                    L.lora_b = torch.zeros((OCt, R), dtype=bf, device=device)   # block-diagonal
+                    L.dlora_b = torch.empty((OCt, R), dtype=f32, device=device)
+                    L.out = torch.empty((BT, OCt), dtype=bf, device=device)
+                    L.dinp = torch.empty((BT, C), dtype=bf, device=device)
+                    L.inp = inp
+                    L.dout = [torch.empty((BT, OCt), dtype=bf, device=device) for _ in range(micro_steps)]
+                    L.members, row = [], 0
+                    for name in names:
+                        L.members.append((specs[name], row, idx))
+                        row += specs[name].OC
+                        idx += 1
+                    self.layers.append(L)
+                    self.groups.append([L])
+                    continue
                 for j, name in enumerate(names):
                     s = specs[name]
                     assert s.C == C
                     L = _Layer(s, idx)
-                    L.group_off, L.group_R = j * r, R
+                    L.rank, L.group_off, L.group_R = r, j * r, R
                     L.a_stack, L.da_stack, L.t_stack, L.u_stack = a_stack, da_stack, t_stack, u_stack
                     L.weight = torch.empty((s.OC, s.C), dtype=bf, device=device)
                     L.lora_a = a_stack[j * r:(j + 1) * r]          # contiguous rows of the stack
@@ -370,9 +403,28 @@ class LoraStack:
             self.generate_inputs()
 
     def seed(self, L, role: int, ms: int = 0) -> int:
-        return synth.tensor_seed(self.config_id, L.index, role, ms) + 100000 * self.seed_offset
+        index = L if isinstance(L, int) else L.index
+        return synth.tensor_seed(self.config_id, index, role, ms) + 100000 * self.seed_offset
+
+    def _generate_fused(self):
+        """The same values as the unfused stack, member by member, in the slices of the group's tensors."""
+        dev, r = self.device, self.r
+        for (L,) in self.groups:
+            first = L.members[0][2]
+            for ms in range(self.micro_steps):
+                L.inp[ms].copy_(synth.normal(self.seed(first, 0, ms), (self.BT, L.spec.C), 1.0, dev))
+            for j, (s, row, index) in enumerate(L.members):
+                L.weight[row:row + s.OC].copy_(synth.normal(self.seed(index, 1), (s.OC, s.C), s.w_std, dev))
+                L.a_stack[j * r:(j + 1) * r].copy_(synth.normal(self.seed(index, 4), (r, s.C), 0.02, dev))
+                L.lora_b[row:row + s.OC, j * r:(j + 1) * r].copy_(
+                    synth.normal(self.seed(index, 5), (s.OC, r), 0.02, dev))
+                for ms in range(self.micro_steps):
+                    L.dout[ms][:, row:row + s.OC].copy_(
+                        synth.normal(self.seed(index, 3, ms), (self.BT, s.OC), 1e-3, dev))
 
     def generate_inputs(self):
+        if self.fused:
+            return self._generate_fused()
         dev = self.device
         for G in self.groups:
             for ms in range(self.micro_steps):  # one input per group, seeded by its first member
@@ -393,8 +445,8 @@ class LoraStack:
 
     def flops_per_micro_step(self) -> int:
         """Forward and dinp through the frozen weight, and the six rank-r products of a projection."""
-        return sum(4 * self.BT * L.spec.C * L.spec.OC + 6 * self.BT * self.r * (L.spec.C + L.spec.OC)
-                   for L in self.layers)
+        specs = [m[0] for L in self.layers for m in L.members] if self.fused else [L.spec for L in self.layers]
+        return sum(4 * self.BT * s.C * s.OC + 6 * self.BT * self.r * (s.C + s.OC) for s in specs)
 
     def calls_per_micro_step(self) -> int:
         return 2 * len(self.layers)
@@ -414,7 +466,7 @@ class LoraStack:
                     hook("fwd", L, True)
                 if self.stacked:
                     nb.nb_lora_linear_forward_stacked(L.out, L.inp[ms], L.weight, None, L.t_stack, L.lora_b, BT,
-                                                      s.C, s.OC, r, L.group_R, L.group_off)
+                                                      s.C, s.OC, L.rank, L.group_R, L.group_off)
                 else:
                     nb.nb_lora_linear_forward(L.out, L.t, L.inp[ms], L.weight, None, L.lora_a, L.lora_b,
                                               self.scale, BT, s.C, s.OC, r)
@@ -432,7 +484,7 @@ class LoraStack:
                 if self.stacked:
                     nb.nb_lora_linear_backward_stacked(L.dinp, L.dlora_b, L.u_stack, L.dout[ms], L.weight,
                                                        L.lora_a, L.lora_b, L.t_stack, self.scale, BT, s.C, s.OC,
-                                                       r, L.group_R, L.group_off, acc)
+                                                       L.rank, L.group_R, L.group_off, acc)
                 else:
                     nb.nb_lora_linear_backward(L.dinp, L.dlora_a, L.dlora_b, L.u, L.dout[ms], L.inp[ms],
                                                L.weight, L.lora_a, L.lora_b, L.t, self.scale, BT, s.C, s.OC,

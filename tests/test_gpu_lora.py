@@ -268,3 +268,45 @@ def test_adapter_stack_driver_two_micro_steps(stacked):
         4 * BT * c * oc + 6 * BT * 16 * (c + oc)
         for c, oc in ((1024, 2048), (1024, 1024), (1024, 1024), (2048, 1024), (1024, 3072), (1024, 3072),
                       (3072, 1024)))
+
+
+def test_adapter_stack_driver_fused_groups():
+    """The projections of a group as one linear layer (weights stacked by rows, B block-diagonal): every
+    member's output columns, adapter gradients and the group's summed input gradient against the oracle
+    of each adapter alone, over two accumulating micro-steps; and the same values as the unfused driver
+    produces from the same seeds."""
+    from paper_2609_28568_b200.stack import LoraStack
+    BT, r = 384, 16
+    st = LoraStack(BT, micro_steps=2, device=DEV, layers=1, fused=True)
+    ref = LoraStack(BT, micro_steps=2, device=DEV, layers=1)
+    st.step()
+    ref.step()
+    torch.cuda.synchronize()
+    assert [L.spec.name for L in st.layers] == ["q_k_v", "o", "gate_up", "down"]
+    assert st.flops_per_micro_step() == ref.flops_per_micro_step()
+    by_name = {L.spec.name: L for L in ref.layers}
+    for (L,) in st.groups:
+        di_sum, slack_sum = 0.0, 0.0
+        for j, (s, row, _) in enumerate(L.members):
+            cols = slice(row, row + s.OC)
+            w, a = f32(L.weight[cols]), f32(L.a_stack[j * r:(j + 1) * r])
+            b = f32(L.lora_b[cols, j * r:(j + 1) * r])
+            U = by_name[s.name]   # the unfused driver's projection: same seeds, same tensors
+            assert torch.equal(L.weight[cols], U.weight) and torch.equal(L.lora_b[cols, j * r:(j + 1) * r], U.lora_b)
+            assert torch.equal(L.dout[1][:, cols], U.dout[1]) and torch.equal(L.inp[1], U.inp[1])
+            # zero blocks beside the member's own: its output takes nothing from the other adapters
+            assert float(L.lora_b[cols].float().abs().sum()) == float(L.lora_b[cols, j * r:(j + 1) * r].float().abs().sum())
+            o_ref = oracle.lora_forward(f32(L.inp[1]), w, None, a, b, st.scale)
+            t_ref, _ = oracle.linear_forward(f32(L.inp[1]), a)
+            check_bf16(L.out[:, cols], o_ref, s.name + " out", extra=_rounding_slack(st.scale * t_ref, b.T))
+            assert torch.equal(L.out[:, cols], U.out), s.name + ": fused and unfused outputs differ"
+            dA = dB = None
+            for ms in range(2):
+                di_ref, dA, dB = oracle.lora_backward(f32(L.dout[ms][:, cols]), f32(L.inp[ms]), w, a, b, st.scale,
+                                                      dA=dA, dB=dB, accumulate=ms > 0)
+            u_ref = oracle.linear_backward(f32(L.dout[1][:, cols]), None, b, want=("dinp",))["dinp"]
+            di_sum = di_sum + di_ref
+            slack_sum = slack_sum + _rounding_slack(st.scale * u_ref, a)
+            check_f32(L.da_stack[j * r:(j + 1) * r], dA, s.name + " dlora_a")
+            check_f32(L.dlora_b[cols, j * r:(j + 1) * r], dB, s.name + " dlora_b")
+        check_bf16(L.dinp, di_sum, L.spec.name + " dinp (sum over the group)", extra=slack_sum)

@@ -17,6 +17,15 @@
 // orders (panel pn starts at tile pn mod tiles), so that at any moment the CTAs work on different
 // rows of B and dB.
 //
+// Optionally a third product rides on the same launch: the panel's contribution to the A gradient,
+//     dA[r, C] (+)= u^T[r, BT] . x[BT, C]                     (contracts BT; fp32, reduce-added)
+// Once a panel's u is final, the epilogue also leaves it (scaled, bf16: the same values it stores) in
+// shared memory in the layout of the t tile, and the CTA streams the panel's rows of x through the
+// same stage ring: each 128 x 128 tile of x, read MN-major exactly like a dy tile in the dB product,
+// times the panel's u gives 128 columns of dA (transposed in TMEM: lanes = columns of x), which the
+// epilogue turns while staging and reduce-adds. The launch of the dA product and its start and end
+// are saved; x is read once, as before.
+//
 // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue (TMEM lane quarter = warp % 4).
 // Every wait is bounded as in gemm_kernel; on expiry the kernel records it and leaves.
 #pragma once
@@ -31,7 +40,8 @@ constexpr uint32_t kUdbBBytes = 16384;  // 128 rows of B (or of t) x 64 columns 
 constexpr uint32_t kUdbOffA = 0;
 constexpr uint32_t kUdbOffB = kUdbStages * kUdbABytes;
 constexpr uint32_t kUdbOffT = kUdbOffB + kUdbStages * kUdbBBytes;
-constexpr uint32_t kUdbOffStg = kUdbOffT + kUdbBBytes;          // 4 warps x 2 boxes of 4 KB
+constexpr uint32_t kUdbOffU = kUdbOffT + kUdbBBytes;            // the panel's u, bf16, laid out like the t tile
+constexpr uint32_t kUdbOffStg = kUdbOffU + kUdbBBytes;          // 4 warps x 2 boxes of 4 KB
 constexpr uint32_t kUdbOffBar = kUdbOffStg + 4 * 2 * 4096;
 constexpr uint32_t kUdbSmemBytes = kUdbOffBar + 256;
 constexpr int kUdbDbBufs = 4;
@@ -42,6 +52,9 @@ struct UdbParams {
     int panels;    // ceil(BT / 128)
     int tiles;     // ceil(OC / 128)
     int want_db;   // 0: only u
+    int want_da;   // 1: also dA (+)= u^T . x, x [BT, C]
+    int C;         // columns of x
+    int xtiles;    // ceil(C / 128)
     float alpha;
     __nv_bfloat16 *u;  // first element of this adapter's column slice of u
     int u_ld;          // elements from one row of u to the next
@@ -54,6 +67,8 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                 const __grid_constant__ CUtensorMap tmB,   // lora_b [OC, r] bf16, 64 x 64 boxes
                 const __grid_constant__ CUtensorMap tmT,   // t slice [BT, r] bf16, 64 x 64 boxes
                 const __grid_constant__ CUtensorMap tmDb,  // dB [OC, r] fp32, 32 x 32 boxes
+                const __grid_constant__ CUtensorMap tmX,   // x [BT, C] bf16, 64 x 64 boxes (want_da)
+                const __grid_constant__ CUtensorMap tmDa,  // dA [r, C] fp32, 32 x 32 boxes (want_da)
                 const UdbParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -74,8 +89,10 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
     const uint32_t u_full = bar0 + 8u * (2 * S + 2), u_empty = bar0 + 8u * (2 * S + 3);
     auto dbfull_bar = [&](int b) { return bar0 + 8u * (2 * S + 4 + b); };
     auto dbempty_bar = [&](int b) { return bar0 + 8u * (2 * S + 4 + NB + b); };
+    // the panel's u in shared memory: written by the four epilogue warps, read by the dA MMAs
+    const uint32_t us_full = bar0 + 8u * (2 * S + 4 + 2 * NB), us_empty = bar0 + 8u * (2 * S + 5 + 2 * NB);
     const uint32_t tmem_slot = bar0 + 240, abort_addr = bar0 + 244;
-    static_assert(8 * (2 * S + 4 + 2 * NB) <= 240, "barrier region");
+    static_assert(8 * (2 * S + 6 + 2 * NB) <= 240, "barrier region");
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -90,8 +107,14 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
             ptx::mbar_init(dbfull_bar(b), 1);
             ptx::mbar_init(dbempty_bar(b), 4);
         }
+        ptx::mbar_init(us_full, 4);   // one arrive per epilogue warp
+        ptx::mbar_init(us_empty, 1);  // the issuer's commit after a panel's last dA MMA
         ptx::st_shared_u32_volatile(abort_addr, 0);
         ptx::fence_barrier_init();
+        if (p.want_da) {
+            ptx::prefetch_tmap(&tmX);
+            ptx::prefetch_tmap(&tmDa);
+        }
         ptx::prefetch_tmap(&tmDy);
         ptx::prefetch_tmap(&tmB);
         ptx::prefetch_tmap(&tmT);
@@ -146,6 +169,23 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                     // B's rows c0..+127 (the k index of the u product), r columns
                     ptx::tma_load_2d(sb, &tmB, full_bar(stage), 0, c0);
                     ptx::tma_load_2d(sb + 8192u, &tmB, full_bar(stage), 0, c0 + 64);
+                    if (++stage == S) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                // the panel's rows of x, tile by tile, through the same ring (no B rows: the panel's
+                // u in shared memory is the other operand)
+                for (int i = 0; i < (p.want_da ? p.xtiles : 0) && ok; ++i) {
+                    ok = wait_barrier(wctx, empty_bar(stage), phase ^ 1u, 110 + stage);
+                    if (!ok) break;
+                    ptx::mbar_expect_tx(full_bar(stage), kUdbABytes);
+                    const uint32_t sa = smem + kUdbOffA + stage * kUdbABytes;
+                    const int c0 = ((i + pn) % p.xtiles) * 128;
+                    ptx::tma_load_2d(sa, &tmX, full_bar(stage), c0, m0);
+                    ptx::tma_load_2d(sa + 8192u, &tmX, full_bar(stage), c0, m0 + 64);
+                    ptx::tma_load_2d(sa + 16384u, &tmX, full_bar(stage), c0 + 64, m0);
+                    ptx::tma_load_2d(sa + 24576u, &tmX, full_bar(stage), c0 + 64, m0 + 64);
                     if (++stage == S) {
                         stage = 0;
                         phase ^= 1u;
@@ -219,6 +259,40 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                 if (!ok) break;
                 ptx::umma_commit<1>(u_full);
                 if (p.want_db) ptx::umma_commit<1>(t_empty);  // t's rows may be replaced once these MMAs are done
+                if (p.want_da) {
+                    // dA_tile^T = x_tile^T . u_panel: the x tile as an MN-major A (as the dy tile in
+                    // the dB product), the panel's u from shared memory as an MN-major B
+                    ok = wait_barrier(wctx, us_full, pphase, 280);
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    const uint64_t udesc = make_smem_desc(smem + kUdbOffU, 8192, 1024);
+                    for (int i = 0; i < p.xtiles; ++i) {
+                        ok = wait_barrier(wctx, full_bar(stage), phase, 310 + stage);
+                        if (!ok) break;
+                        ok = wait_barrier(wctx, dbempty_bar(buf), bphase ^ 1u, 290 + buf);
+                        if (!ok) break;
+                        ptx::tc_fence_after();
+                        const uint32_t sa = smem + kUdbOffA + stage * kUdbABytes;
+                        const uint32_t d_tmem = tmem_base + 64u + static_cast<uint32_t>(buf) * 64u;
+                        const uint64_t adesc = make_smem_desc(sa, 16384, 1024);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            ptx::umma_bf16<1>(d_tmem, adesc + static_cast<uint64_t>(k * (2048u >> 4)),
+                                              udesc + static_cast<uint64_t>(k * (2048u >> 4)), idesc_db, k > 0 ? 1u : 0u);
+                        ptx::umma_commit<1>(empty_bar(stage));
+                        ptx::umma_commit<1>(dbfull_bar(buf));
+                        if (++buf == NB) {
+                            buf = 0;
+                            bphase ^= 1u;
+                        }
+                        if (++stage == S) {
+                            stage = 0;
+                            phase ^= 1u;
+                        }
+                    }
+                    if (!ok) break;
+                    ptx::umma_commit<1>(us_empty);  // the panel's u in shared memory may be replaced
+                }
             }
         }
     } else {
@@ -290,9 +364,30 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
             if (!ok) break;
             ptx::tc_fence_after();
             const long long row = static_cast<long long>(pn) * 128 + q * 32 + lane;
-            for (int c = 0; c < p.r; c += 32) {
+            if (p.want_da) {  // the previous panel's dA MMAs have read the shared copy of its u
+                bool w2 = true;
+                if (lane == 0) w2 = wait_barrier(wctx_epi, us_empty, pphase ^ 1u, 460);
+                ok = __shfl_sync(0xffffffffu, w2 ? 1 : 0, 0) != 0;
+                if (!ok) break;
+            }
+            for (int c = 0; c < (p.want_da ? 64 : p.r); c += 32) {
                 uint32_t r32[32];
                 ptx::tmem_ld_32x32_wait(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c), r32);
+                if (p.want_da) {
+                    // row q*32 + lane of the u tile: 64 bf16 = eight 16-byte pieces, 128-byte swizzle
+                    // (columns beyond r are the zeros the TMA filled B with)
+                    const uint32_t urow = smem + kUdbOffU + static_cast<uint32_t>(q * 32 + lane) * 128u;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t piece = static_cast<uint32_t>((c >> 3) + i);
+                        ptx::st_shared_v4(urow + ((piece ^ sw) << 4),
+                                          ptx::pack_bf16x2(p.alpha * __uint_as_float(r32[i * 8 + 0]), p.alpha * __uint_as_float(r32[i * 8 + 1])),
+                                          ptx::pack_bf16x2(p.alpha * __uint_as_float(r32[i * 8 + 2]), p.alpha * __uint_as_float(r32[i * 8 + 3])),
+                                          ptx::pack_bf16x2(p.alpha * __uint_as_float(r32[i * 8 + 4]), p.alpha * __uint_as_float(r32[i * 8 + 5])),
+                                          ptx::pack_bf16x2(p.alpha * __uint_as_float(r32[i * 8 + 6]), p.alpha * __uint_as_float(r32[i * 8 + 7])));
+                    }
+                }
+                if (c >= p.r) continue;
                 if (row < p.BT) {
                     __nv_bfloat16 *dst = p.u + row * p.u_ld + c;
 #pragma unroll
@@ -308,10 +403,59 @@ lora_udb_kernel(const __grid_constant__ CUtensorMap tmDy,  // dy [BT, OC] bf16, 
                     }
                 }
             }
+            if (p.want_da) ptx::fence_proxy_async_smem();  // the MMAs read the shared copy through the async proxy
             ptx::tc_fence_before();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(u_empty);
+            if (lane == 0) {
+                if (p.want_da) ptx::mbar_arrive(us_full);
+                ptx::mbar_arrive(u_empty);
+            }
             __syncwarp();
+            if (p.want_da) {
+                // 128 columns of dA per x tile, transposed in TMEM: this warp's lanes are 32 columns c of
+                // x, its registers the rows j of dA. Staged as box row j, column lane (a warp-wide store
+                // fills one 128-byte row: no bank conflicts), then reduce-added as a 32 x 32 box.
+                for (int i = 0; i < p.xtiles; ++i) {
+                    bool w3 = true;
+                    if (lane == 0) w3 = wait_barrier(wctx_epi, dbfull_bar(buf), bphase, 470 + buf);
+                    ok = __shfl_sync(0xffffffffu, w3 ? 1 : 0, 0) != 0;
+                    if (!ok) break;
+                    ptx::tc_fence_after();
+                    const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + 64u +
+                                           static_cast<uint32_t>(buf) * 64u;
+                    for (int jb = 0; jb < p.r; jb += 32) {
+                        uint32_t r32[32];
+                        ptx::tmem_ld_32x32_wait(t_acc + static_cast<uint32_t>(jb), r32);
+                        const uint32_t fb = stg + (box & 1u) * 4096u;
+                        ++box;
+                        ptx::bulk_wait_group_read<1>();
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            ptx::st_shared_u32(fb + static_cast<uint32_t>(j) * 128u +
+                                                   (((static_cast<uint32_t>(lane) >> 2) ^ static_cast<uint32_t>(j & 7)) << 4) +
+                                                   (static_cast<uint32_t>(lane) & 3u) * 4u,
+                                               r32[j]);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (ptx::elect_one()) {
+                            const int x = ((i + pn) % p.xtiles) * 128 + q * 32;
+                            if (x < p.C) ptx::tma_reduce_add_2d(&tmDa, fb, x, jb);
+                            ptx::bulk_commit_group();
+                        }
+                        __syncwarp();
+                    }
+                    ptx::tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(dbempty_bar(buf));
+                    __syncwarp();
+                    if (++buf == NB) {
+                        buf = 0;
+                        bphase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+            }
         }
         ptx::bulk_wait_group<0>();
         __syncwarp();

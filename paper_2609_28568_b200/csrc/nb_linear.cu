@@ -483,9 +483,11 @@ int run_wgrad_f32(DeviceState &s, const void *dz, const void *inp, void *dweight
 
 // u = bf16(scale * dy . B) and dB (+)= dy^T . t of one adapted projection from one pass over dy
 // (lora_udb_sm100.cuh). u and t may be column slices of wider tensors (row strides u_ld, t_ld).
+// x and dlora_a both non-NULL: the A gradient dlora_a [r, C] (+)= u^T . x rides on the same launch
+// (only with the whole of u in one call: u_ld == r).
 int launch_lora_udb(DeviceState &s, const void *dy, const void *lora_b, const void *t, uint64_t t_ld, void *dlora_b,
                     void *u, uint64_t u_ld, float scale, int64_t BT, int64_t OC, int64_t r, int accumulate,
-                    cudaStream_t stream)
+                    cudaStream_t stream, const void *x = nullptr, void *dlora_a = nullptr, int64_t C = 0)
 {
     static bool attr_set[kMaxDevices] = {};
     int dev = 0;
@@ -495,14 +497,25 @@ int launch_lora_udb(DeviceState &s, const void *dy, const void *lora_b, const vo
                                      static_cast<int>(kUdbSmemBytes)));
         attr_set[dev] = true;
     }
-    CUtensorMap tDy, tB, tT, tDb;
+    const bool want_da = x != nullptr && dlora_a != nullptr;
+    CUtensorMap tDy, tB, tT, tDb, tX, tDa;
     int rc;
     if ((rc = get_tmap(s, &tDy, dy, BT, OC, 0, 64)) != NB_OK) return rc;
     if ((rc = get_tmap(s, &tB, lora_b, OC, r, 0, 64)) != NB_OK) return rc;
     if ((rc = get_tmap(s, &tT, t, BT, r, 0, 64, t_ld)) != NB_OK) return rc;
     if ((rc = get_tmap(s, &tDb, dlora_b, OC, r, 1, 32)) != NB_OK) return rc;
+    if (want_da) {
+        if ((rc = get_tmap(s, &tX, x, BT, C, 0, 64)) != NB_OK) return rc;
+        if ((rc = get_tmap(s, &tDa, dlora_a, r, C, 1, 32)) != NB_OK) return rc;
+    } else {
+        tX = tDy;   // never dereferenced
+        tDa = tDb;
+    }
     // every panel reduce-adds its share, so a fresh gradient starts from zero
-    if (!accumulate) NB_CUDA(cudaMemsetAsync(dlora_b, 0, static_cast<size_t>(OC * r) * 4, stream));
+    if (!accumulate) {
+        NB_CUDA(cudaMemsetAsync(dlora_b, 0, static_cast<size_t>(OC * r) * 4, stream));
+        if (want_da) NB_CUDA(cudaMemsetAsync(dlora_a, 0, static_cast<size_t>(r * C) * 4, stream));
+    }
     UdbParams p;
     memset(&p, 0, sizeof(p));
     p.BT = static_cast<int>(BT);
@@ -511,6 +524,9 @@ int launch_lora_udb(DeviceState &s, const void *dy, const void *lora_b, const vo
     p.panels = static_cast<int>((BT + 127) / 128);
     p.tiles = static_cast<int>((OC + 127) / 128);
     p.want_db = 1;
+    p.want_da = want_da ? 1 : 0;
+    p.C = static_cast<int>(C);
+    p.xtiles = want_da ? static_cast<int>((C + 127) / 128) : 0;
     p.alpha = scale;
     p.u = static_cast<__nv_bfloat16 *>(u);
     p.u_ld = static_cast<int>(u_ld);
@@ -526,7 +542,7 @@ int launch_lora_udb(DeviceState &s, const void *dy, const void *lora_b, const vo
     attrs[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attrs;
     cfg.numAttrs = dependent_launch_allowed(stream) ? 1 : 0;
-    NB_CUDA(cudaLaunchKernelEx(&cfg, lora_udb_kernel, tDy, tB, tT, tDb, p));
+    NB_CUDA(cudaLaunchKernelEx(&cfg, lora_udb_kernel, tDy, tB, tT, tDb, tX, tDa, p));
     ++g_launches;
     return NB_OK;
 }
@@ -1087,11 +1103,14 @@ int nb_lora_linear_backward(void *dinp, void *dlora_a, void *dlora_b, void *u, c
     }
     GemmArgs a;
     static const bool fused_udb = env_int("NB_LORA_FUSED", 1) != 0;
-    if (fused_udb && dlora_b) {  // u and dB from one pass over dout
+    static const bool fused_da = env_int("NB_LORA_FUSED_DA", 1) != 0;
+    if (fused_udb && dlora_b) {  // u and dB from one pass over dout; dA from one pass over inp in the same launch
+        const bool with_da = fused_da && dlora_a != nullptr;
         if ((rc = launch_lora_udb(*s, dout, lora_b, t, 0, dlora_b, u, static_cast<uint64_t>(r), scale, BT, OC, r,
-                                  accumulate, stream)) != NB_OK)
+                                  accumulate, stream, with_da ? inp : nullptr, with_da ? dlora_a : nullptr, C)) != NB_OK)
             return rc;
         dlora_b = nullptr;
+        if (with_da) dlora_a = nullptr;
     } else {
         memset(&a, 0, sizeof(a));  // u = scale * dout . B   (B [OC, r] read as an MN-major operand)
         a.A = dout; a.a_rows = BT; a.a_cols = OC;

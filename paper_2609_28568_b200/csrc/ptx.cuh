@@ -356,6 +356,11 @@ __device__ __forceinline__ void st_shared_u32_volatile(uint32_t addr, uint32_t v
     asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
+__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
 // ------------------------------------------------------------------ packed fp32 math (two lanes)
 // sm_100 executes fma / mul / add on pairs of fp32 held in a 64-bit register: half the issue slots
 // of the scalar forms, which is what the activation epilogues are short of.

@@ -481,7 +481,13 @@ class LoraStack:
                 s = L.spec
                 if hook:
                     hook("bwd", L, True)
-                if self.stacked:
+                if self.fused:
+                    # the group is one adapter of rank R: u and dB from one pass over dout, dA from one
+                    # pass over the input in the same launch, then the dinp product
+                    nb.nb_lora_linear_backward(L.dinp, L.da_stack, L.dlora_b, L.u_stack, L.dout[ms], L.inp[ms],
+                                               L.weight, L.a_stack, L.lora_b, L.t_stack, self.scale, BT, s.C, s.OC,
+                                               L.rank, acc)
+                elif self.stacked:
                     nb.nb_lora_linear_backward_stacked(L.dinp, L.dlora_b, L.u_stack, L.dout[ms], L.weight,
                                                        L.lora_a, L.lora_b, L.t_stack, self.scale, BT, s.C, s.OC,
                                                        L.rank, L.group_R, L.group_off, acc)
@@ -491,7 +497,7 @@ class LoraStack:
                                                r, acc)
                 if hook:
                     hook("bwd", L, False)
-            if self.stacked:
+            if self.stacked and not self.fused:
                 L0 = G[0]
                 nb.nb_lora_da_stacked(L0.da_stack, L0.u_stack, L0.inp[ms], BT, L0.spec.C, L0.group_R, acc)
 

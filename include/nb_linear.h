@@ -207,7 +207,17 @@ int nb_ce_backward(void *dlogits, const void *logits, const void *lse, const voi
  * dinp, dlora_a, dlora_b may be NULL (skipped); accumulate as in nb_linear_backward. t and u are
  * rounded to bf16 once each (they are tensor-core operands); everything else follows the
  * conventions at the top of this file. When dlora_b is asked for, u and dlora_b come out of one
- * kernel that reads dout once (both products are bound by that read).
+ * kernel that reads dout once (both products are bound by that read); when dlora_a is asked for
+ * as well, the same launch also reads inp once and forms dlora_a. Both gradients are summed by
+ * reduce-adds of per-row-panel partial sums, in no fixed order.
+ *
+ * Projections that share an input and are laid out as one layer (a qkv or a gate_up projection:
+ * weights stacked by rows) can use these two calls as they are, with r = the sum of the members'
+ * ranks (<= 64): lora_a = the members' A matrices stacked by rows, lora_b [sum of OC, r] = their B
+ * matrices as diagonal blocks and zeros elsewhere. Every member's columns of out, its rows of
+ * dlora_a and its diagonal block of dlora_b then equal what the member alone would give, dinp is
+ * the sum of the members' input gradients, and the other blocks of dlora_b hold values that belong
+ * to no parameter.
  */
 int nb_lora_linear_forward(void *out, void *t, const void *inp, const void *weight, const void *bias,
                            const void *lora_a, const void *lora_b, float scale, int64_t BT,
